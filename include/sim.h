@@ -1,0 +1,138 @@
+/*
+ * sim.h -- C ABI of the batched environment-stepping library (CUDA, sm_100a).
+ *
+ * The problem, as the paper states it: N simulator instances advance in parallel on the
+ * GPU ("GPU vectorization", Section 3) and K simulator steps run inside one kernel launch
+ * with the simulator state cached on chip ("simulator kernel fusion", Section 4).  Each
+ * step here is: pick an action (uniform random, a small MLP, or given by the caller),
+ * advance the physics, compute reward and done, auto-reset finished envs, and append to a
+ * trajectory buffer.  N envs never interact.
+ *
+ * Conventions for every call
+ *   - Return value: 0 (SIM_OK) or a negative SIM_E* code.  Nothing throws or aborts.
+ *     Argument errors are detected on the host before any work is enqueued.
+ *   - Pointers named d_* / out_* are DEVICE pointers owned by the caller; they must stay
+ *     valid until the work enqueued by the call has finished.  Pointers named h_* are
+ *     HOST pointers.  The library never frees or keeps a caller pointer.
+ *   - The handle and its internal buffers (state [N,S] fp32 row-major, ep_len [N] u32,
+ *     reset_count [N] u32) are owned by the library: sim_create allocates, sim_destroy frees.
+ *   - Except sim_create / sim_destroy / sim_rollout_host, calls only enqueue work on the
+ *     handle's stream and return; the caller synchronises the stream.
+ *   - All floating point is IEEE binary32 with a fixed operation order, so results are
+ *     reproducible bit for bit for a given (seed, env index, step index), whatever K is.
+ *   - Random numbers: Philox4x32-10 keyed by the seed.  Action word of (env, t) = word
+ *     (t mod 4) of the block with counter (env, t div 4, 0, 0).  State draw r of an env
+ *     (r = 0 at reset, r = reset_count after the r-th auto-reset) uses counters
+ *     (env, r, 1, j) for elements 4j..4j+3.
+ *   - Action encoding: CartPole 0 = push left (-10 N), 1 = push right; Acrobot 0,1,2 =
+ *     torque -1,0,+1; synthetic 0,1 = a = -1,+1.  Out-of-range bytes: CartPole and
+ *     synthetic use (a != 0); Acrobot clamps to [0,2].
+ */
+#ifndef PAPER_2207_07736_SIM_H
+#define PAPER_2207_07736_SIM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sim sim_t;   /* opaque */
+
+enum { SIM_CARTPOLE = 0, SIM_ACROBOT = 1, SIM_SYNTH = 2 };
+enum { SIM_OK = 0, SIM_EINVAL = -1, SIM_ENOMEM = -2, SIM_ECUDA = -3, SIM_ESTATE = -4 };
+
+#define SIM_POLICY_PARAM_COUNT 4610   /* W1[64][4] b1[64] W2[64][64] b2[64] W3[2][64] b3[2], rows = output units */
+
+/*
+ * sim_create -- make N simulator instances on the current CUDA device (Section 3: "N
+ * simulator instances in parallel"; Section 2.2: CartPole state of S = 4 floats; Section
+ * 4.2: the state-size factor S of the synthetic simulator).
+ *   out       receives the handle.
+ *   env_kind  SIM_CARTPOLE | SIM_ACROBOT | SIM_SYNTH.
+ *   n_envs    1 .. 2^32-1.
+ *   state_dim 4 for CartPole/Acrobot; a power of two in [4, 4096] for SIM_SYNTH.
+ *   seed      Philox key.
+ * Allocates device memory, then enqueues the initial-state draw (like sim_reset) on the
+ * default stream and waits for it.  Errors: SIM_EINVAL, SIM_ENOMEM, SIM_ECUDA.
+ */
+int sim_create(sim_t **out, int env_kind, int64_t n_envs, int state_dim, uint64_t seed);
+
+/* sim_destroy -- wait for the handle's stream, free everything.  NULL is SIM_EINVAL. */
+int sim_destroy(sim_t *s);
+
+/* sim_set_stream -- use this cudaStream_t (passed as void*) for all later work; NULL = default stream. */
+int sim_set_stream(sim_t *s, void *cuda_stream);
+
+/* sim_set_env_offset -- global index of this handle's env 0 (default 0).  Random draws are keyed by
+ * offset + local index, so handles that own disjoint ranges of one global population reproduce the
+ * single-handle result exactly (sharding across GPUs needs no exchange: envs never interact).
+ * offset + n_envs must not exceed 2^32.  Takes effect at the next sim_reset. */
+int sim_set_env_offset(sim_t *s, uint64_t env_offset);
+
+/* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env. */
+int sim_reset(sim_t *s);
+
+/*
+ * sim_step -- one step of every env with caller-given actions: the step() state
+ * transition of Section 3.2, vectorised over N (one kernel launch).
+ *   d_actions  [N] int8 action indices.
+ *   d_next_obs [N,S] fp32, state after the step and after auto-reset (may be NULL).
+ *   d_rew      [N] fp32 (may be NULL).      d_done [N] u8 (may be NULL).
+ * Advances t by one.
+ */
+int sim_step(sim_t *s, const int8_t *d_actions, float *d_next_obs, float *d_rew, uint8_t *d_done);
+
+/*
+ * sim_rollout -- T steps of every env in ceil(T / K_fused) kernel launches; inside one
+ * launch the state lives in registers / shared memory (Section 4, "K simulator steps are
+ * executed in a single fused GPU kernel launch").  K_fused = 1 is plain GPU vectorization.
+ *   T >= 1, K_fused >= 1 (values above T are clamped to T).
+ *   d_policy_params  NULL = uniform random actions; else SIM_POLICY_PARAM_COUNT floats of
+ *                    the 4-64-64-2 tanh MLP whose softmax is sampled with the action word
+ *                    (CartPole only; SIM_EINVAL for the other kinds).
+ *   out_obs  [T,N,S] fp32: state each env's policy saw at step t (before the step).
+ *   out_act  [T,N] int8.   out_rew [T,N] fp32.   out_done [T,N] u8.
+ *   Any of the four may be NULL and is then not written.
+ * Results do not depend on K_fused.  Advances t by T.
+ */
+int sim_rollout(sim_t *s, int T, int K_fused, const float *d_policy_params,
+                float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done);
+
+/*
+ * sim_rollout_host -- the same rollout with HOST buffers, for callers that consume the
+ * trajectory on the CPU.  h_policy_params (NULL or SIM_POLICY_PARAM_COUNT floats) is
+ * copied to the device; the trajectory is produced in chunks of K_fused steps into
+ * library-owned device staging buffers and copied to the h_* arrays (same shapes as in
+ * sim_rollout, each may be NULL) while the next chunk is being computed.  Pinned host
+ * memory gives the best copy rate; pageable memory works.  Blocks until all copies are
+ * done.  Staging buffers (two chunks) are allocated on first use and kept by the handle;
+ * SIM_ENOMEM if they do not fit.
+ */
+int sim_rollout_host(sim_t *s, int T, int K_fused, const float *h_policy_params,
+                     float *h_obs, int8_t *h_act, float *h_rew, uint8_t *h_done);
+
+/* Inspection and checkpoint hooks: copy state / counters out of or into the handle
+ * (device pointers; d_* may be NULL to skip one).  h_t is a host pointer. */
+int sim_get_state(sim_t *s, float *d_state /* [N,S] */);
+int sim_set_state(sim_t *s, const float *d_state /* [N,S] */);
+int sim_get_counters(sim_t *s, uint32_t *d_ep_len, uint32_t *d_reset_count, uint64_t *h_t);
+int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t *d_reset_count, uint64_t t);
+
+/* sim_policy_logits -- logits of the MLP for M observations (no sampling, no stepping).
+ *   d_obs [M,4] fp32, d_params SIM_POLICY_PARAM_COUNT fp32, d_logits [M,2] fp32.  s may be
+ *   any live handle (it provides the stream). */
+int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits);
+
+/* sim_launch_count -- kernels launched by this handle since creation (for launch accounting). */
+int64_t sim_launch_count(sim_t *s);
+
+/* sim_strerror -- static string for a SIM_* code.  sim_last_cuda_error -- the cudaError_t
+ * behind the most recent SIM_ECUDA of this handle (0 if none). */
+const char *sim_strerror(int code);
+int sim_last_cuda_error(sim_t *s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

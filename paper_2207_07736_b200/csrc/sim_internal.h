@@ -1,0 +1,58 @@
+// Host-side declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+#include "sim_math.cuh"
+
+namespace simk {
+
+enum : int { POLICY_RANDOM = 0, POLICY_GIVEN = 1, POLICY_MLP = 2 };
+
+// Arguments of one launch over envs with a 4-float state (CartPole, Acrobot).
+// Output pointers are already advanced to the row of the launch's first step.
+struct S4Args {
+    float4 *state;            // [n]
+    uint32_t *ep_len;         // [n]
+    uint32_t *reset_count;    // [n]
+    uint32_t n;               // envs in this handle
+    uint32_t env_offset;      // global index of env 0
+    uint32_t tb0;             // (t0 >> 2) truncated to 32 bits: Philox counter word of the first action block
+    int phase;                // t0 & 3
+    int K;                    // steps in this launch
+    float4 *out_obs;          // [K, n] or nullptr
+    int8_t *out_act;          // [K, n] or nullptr
+    float *out_rew;           // [K, n] or nullptr
+    uint8_t *out_done;        // [K, n] or nullptr
+    const int8_t *actions;    // [n], POLICY_GIVEN only
+    float4 *next_obs;         // [n] post-step state, POLICY_GIVEN only (nullable)
+    const float *params;      // MLP parameters, POLICY_MLP only
+    RoundKeys rk;
+};
+
+// Arguments of one launch of the synthetic S-float simulator.
+struct SynthArgs {
+    float *state;             // [n, S]
+    uint32_t *ep_len;
+    uint32_t *reset_count;
+    uint32_t n;
+    uint32_t env_offset;
+    uint32_t tb0;
+    int phase;
+    int K;
+    float *out_obs;           // [K, n, S] or nullptr
+    int8_t *out_act;
+    float *out_rew;
+    uint8_t *out_done;
+    const int8_t *actions;    // [n] or nullptr (given-action step, K == 1)
+    float *next_obs;          // [n, S] or nullptr
+    RoundKeys rk;
+};
+
+// Launchers (each returns the launch error, enqueues on `st`, never synchronises).
+cudaError_t launch_reset(int env_kind, int S, float *state, uint32_t *ep_len, uint32_t *reset_count,
+                         uint32_t n, uint32_t env_offset, const RoundKeys &rk, cudaStream_t st);
+cudaError_t launch_s4(int env_kind, int policy, const S4Args &a, cudaStream_t st);
+cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st);
+cudaError_t launch_policy_logits(const float *obs, int64_t M, const float *params, float *logits, cudaStream_t st);
+
+}  // namespace simk

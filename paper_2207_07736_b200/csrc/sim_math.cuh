@@ -1,0 +1,115 @@
+// Device arithmetic of the environment-stepping kernels (sm_100a).
+//
+// Every floating-point operation is written with an explicit round-to-nearest intrinsic
+// (__fadd_rn, __fmul_rn, __fmaf_rn, __fdiv_rn, __frcp_rn) so that the compiler can neither
+// contract nor reorder it: results are identical bit for bit on every launch shape and do
+// not depend on compiler flags.  Elementary functions are fixed polynomial evaluations
+// (no libm, no fast-math approximations).
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace simk {
+
+__device__ __forceinline__ float fbits(uint32_t b) { return __uint_as_float(b); }
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10.  The ten round keys depend only on the seed, so the host expands them once and
+// they arrive as kernel parameters (constant-bank operands of the xor instructions).
+// ---------------------------------------------------------------------------------------------
+struct RoundKeys { uint32_t k[10][2]; };
+
+__device__ __forceinline__ uint4 philox(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const RoundKeys &rk)
+{
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+        uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        uint32_t n0 = hi1 ^ c1 ^ rk.k[r][0];
+        uint32_t n2 = hi0 ^ c3 ^ rk.k[r][1];
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// u in [0, 1 - 2^-24]: top 24 bits, exact.
+__device__ __forceinline__ float uniform01(uint32_t w) { return __fmul_rn(__uint2float_rn(w >> 8), fbits(0x33800000u)); }
+
+// lo + width*u with a single rounding.
+__device__ __forceinline__ float uniform_range(uint32_t w, float width, float lo) { return __fmaf_rn(uniform01(w), width, lo); }
+
+// ---------------------------------------------------------------------------------------------
+// Round-to-nearest-even to an integer by adding 1.5*2^23: valid for |t| < 2^22.  `neg_k` is the
+// negated integer (exact, and +0 when the integer is 0), `bits` carries the integer in its low
+// mantissa bits (two's complement), so no float->int conversion instruction is needed.
+// ---------------------------------------------------------------------------------------------
+constexpr float kRoundMagic = 12582912.0f;
+
+// sin and cos of x (|x| < 1e6): three-term Cody-Waite reduction by pi/2, degree-9 / degree-10
+// Taylor polynomials with fused multiply-adds, quadrant fix-up by sign-bit arithmetic.
+__device__ __forceinline__ void sincos_s(float x, float &sn, float &cs)
+{
+    const float t = __fmul_rn(x, fbits(0x3F22F983u));           // x * 2/pi
+    const float nb = __fadd_rn(t, kRoundMagic);
+    const float nk = __fsub_rn(kRoundMagic, nb);                 // -k
+    const uint32_t q = __float_as_uint(nb);
+    float r = __fmaf_rn(nk, fbits(0x3FC90FDBu), x);
+    r = __fmaf_rn(nk, fbits(0xB33BBD2Eu), r);
+    r = __fmaf_rn(nk, fbits(0xA6F72CEDu), r);
+    const float r2 = __fmul_rn(r, r);
+    float p = __fmaf_rn(fbits(0x3638EF1Du), r2, fbits(0xB9500D01u));
+    p = __fmaf_rn(p, r2, fbits(0x3C088889u));
+    p = __fmaf_rn(p, r2, fbits(0xBE2AAAABu));
+    const float S = __fmaf_rn(p, __fmul_rn(r2, r), r);
+    float c = __fmaf_rn(fbits(0xB493F27Eu), r2, fbits(0x37D00D01u));
+    c = __fmaf_rn(c, r2, fbits(0xBAB60B61u));
+    c = __fmaf_rn(c, r2, fbits(0x3D2AAAABu));
+    c = __fmaf_rn(c, r2, -0.5f);
+    const float C = __fmaf_rn(c, r2, 1.0f);
+    const bool odd = q & 1u;
+    const float a = odd ? C : S;
+    const float b = odd ? S : C;
+    sn = __uint_as_float(__float_as_uint(a) ^ ((q & 2u) << 30));
+    cs = __uint_as_float(__float_as_uint(b) ^ (((q + 1u) & 2u) << 30));
+}
+
+__device__ __forceinline__ float sin_s(float x) { float s, c; sincos_s(x, s, c); return s; }
+__device__ __forceinline__ float cos_s(float x) { float s, c; sincos_s(x, s, c); return c; }
+
+// exp(y) for y already inside [-87, 88].
+__device__ __forceinline__ float exp_core(float y)
+{
+    const float t = __fmul_rn(y, fbits(0x3FB8AA3Bu));           // y * log2(e)
+    const float nb = __fadd_rn(t, kRoundMagic);
+    const float nn = __fsub_rn(kRoundMagic, nb);                 // -n
+    float r = __fmaf_rn(nn, fbits(0x3F317218u), y);
+    r = __fmaf_rn(nn, fbits(0xB102E308u), r);
+    float p = __fmaf_rn(fbits(0x39500D01u), r, fbits(0x3AB60B61u));
+    p = __fmaf_rn(p, r, fbits(0x3C088889u));
+    p = __fmaf_rn(p, r, fbits(0x3D2AAAABu));
+    p = __fmaf_rn(p, r, fbits(0x3E2AAAABu));
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    const float scale = __uint_as_float((__float_as_uint(nb) << 23) + 0x3F800000u);   // 2^n
+    return __fmul_rn(p, scale);
+}
+
+__device__ __forceinline__ float exp_s(float y) { return exp_core(fminf(fmaxf(y, -87.0f), 88.0f)); }
+
+// tanh(x) = sign(x) * (1 - 2/(exp(2|x|)+1)), saturating to 1 above |x| = 9 (whatever exp_core
+// returns for larger arguments is discarded by the select).
+// 2/d is twice the correctly rounded reciprocal (scaling by two is exact), so the final
+// subtraction is one fused multiply-add.
+__device__ __forceinline__ float tanh_s(float x)
+{
+    const float a = fabsf(x);
+    const float e = exp_core(__fadd_rn(a, a));                  // the clamp of exp is inactive for a <= 9
+    const float d = __fadd_rn(e, 1.0f);
+    float t = __fmaf_rn(-2.0f, __frcp_rn(d), 1.0f);
+    t = (a > 9.0f) ? 1.0f : t;
+    return copysignf(t, x);
+}
+
+}  // namespace simk

@@ -1,0 +1,197 @@
+"""GPU-vs-oracle parity through the C ABI, bit for bit (actions, flags, counters, fp32 states),
+at sizes the oracle finishes in seconds: several CTAs, a ragged tail, K that does not divide T,
+launches that start at every phase of the 4-step action block."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2207_07736_b200 import binding, inputs
+from gpu_common import assert_same_bits, compare_rollout, to_np, torch_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+def run_pair(kind, n, T, K, S=4, seed=0, params=None, pre=None):
+    torch = torch_cuda()
+    sim = binding.Sim(kind, n, S, seed)
+    orc = oracle.OracleSim(kind, n, S, seed)
+    if pre is not None:
+        pre(sim, orc, torch)
+    d_params = None if params is None else torch.from_numpy(params).cuda()
+    out = sim.rollout(T, K, d_params)
+    torch.cuda.synchronize()
+    ref = orc.rollout(T, policy_params=params)
+    compare_rollout(out, sim, ref, orc, what="kind%d n%d T%d K%d S%d" % (kind, n, T, K, S))
+    return sim, out
+
+
+def test_cfg1_cartpole_small_exact():
+    w = inputs.WORKLOADS["cfg1"]
+    sim, out = run_pair(w.env_kind, w.n_envs, w.T, 1, seed=w.seed)
+    assert sim.launches == 1 + w.T                       # one reset kernel + one launch per step
+    assert float(out["rew"].min()) == 1.0 and int(out["done"].sum()) > 0
+
+
+@pytest.mark.parametrize("K", [1, 3, 7, 10, 64, 157, 1000])
+def test_cartpole_any_k_ragged(K):
+    sim, _ = run_pair(oracle.CARTPOLE, 1000, 157, K, seed=3)
+    assert sim.launches == 1 + -(-157 // min(K, 157))
+
+
+@pytest.mark.parametrize("K", [1, 50, 500, 1100])
+def test_acrobot_any_k(K):
+    n, T = (64, 120) if K == 1 else (300, 1100)          # 1100 steps cross the 500-step limit twice
+    sim, out = run_pair(oracle.ACROBOT, n, T, K, seed=5)
+    if T > 500:
+        assert int(out["done"][499].sum()) > n // 2
+
+
+def test_acrobot_wrap_and_clip_states():
+    def pre(sim, orc, torch):
+        rng = np.random.default_rng(0)
+        st = (rng.uniform(-1, 1, (sim.n, 4)) * np.array([3.14, 3.14, 12.5, 28.0])).astype(np.float32)
+        orc.state[:] = st
+        sim.set_state(torch.from_numpy(st).cuda())
+    run_pair(oracle.ACROBOT, 257, 30, 30, seed=1, pre=pre)
+
+
+@pytest.mark.parametrize("S", [4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096])
+def test_synth_all_shapes(S):
+    n = 37 if S <= 512 else 5
+
+    def pre(sim, orc, torch):
+        st = orc.state.copy()
+        st[::3] = 2.02                                   # every third env terminates on the first step
+        st[1::7] *= 2.2                                  # some drift over the threshold later
+        orc.state[:] = st
+        sim.set_state(torch.from_numpy(st).cuda())
+    for K in (1, 5, 22):
+        sim, out = run_pair(oracle.SYNTH, n, 22, K, S=S, seed=2, pre=pre)
+        assert int(out["done"][0].sum()) >= n // 3
+
+
+def test_synth_larger_batch_spans_many_ctas():
+    run_pair(oracle.SYNTH, 3001, 9, 4, S=4, seed=8)
+    run_pair(oracle.SYNTH, 1025, 9, 9, S=64, seed=8)
+    run_pair(oracle.SYNTH, 70, 6, 3, S=4096, seed=8)
+
+
+@pytest.mark.parametrize("bias_std", [0.0, 0.5])
+@pytest.mark.parametrize("K", [1, 9, 60])
+def test_mlp_policy(K, bias_std):
+    p = inputs.mlp_params(1, bias_std)
+    sim, out = run_pair(oracle.CARTPOLE, 300, 60, K, seed=4, params=p)
+    frac0 = float((out["act"] == 0).float().mean())
+    assert 0.05 < frac0 < 0.95
+
+
+def test_mlp_zero_params_equal_random_policy():
+    torch = torch_cuda()
+    z = torch.zeros(inputs.MLP_PARAM_COUNT, dtype=torch.float32, device="cuda")
+    a = binding.Sim(oracle.CARTPOLE, 500, 4, 9)
+    b = binding.Sim(oracle.CARTPOLE, 500, 4, 9)
+    ra, rb = a.rollout(80, 80), b.rollout(80, 16, z)
+    for k in ("obs", "act", "rew", "done"):
+        assert torch.equal(ra[k], rb[k])
+
+
+def test_policy_logits_entry_point():
+    torch = torch_cuda()
+    rng = np.random.default_rng(0)
+    obs = (rng.uniform(-1, 1, (1000, 4)) * np.array([2.4, 3, 0.21, 3])).astype(np.float32)
+    sim = binding.Sim(oracle.CARTPOLE, 8)
+    for seed, bias in ((1, 0.0), (7, 0.3)):
+        p = inputs.mlp_params(seed, bias)
+        got = to_np(sim.policy_logits(torch.from_numpy(obs).cuda(), torch.from_numpy(p).cuda()))
+        want = np.stack([oracle.mlp_logits(p, o) for o in obs])
+        assert np.abs(got - want).max() <= 1e-5          # the stated tolerance
+        assert_same_bits(got, want, "logits")            # and in fact identical
+
+
+@pytest.mark.parametrize("kind,S,nact", [(oracle.CARTPOLE, 4, 2), (oracle.ACROBOT, 4, 3), (oracle.SYNTH, 64, 2), (oracle.SYNTH, 2048, 2)])
+def test_step_with_given_actions(kind, S, nact):
+    torch = torch_cuda()
+    n, T = 203, 40
+    sim = binding.Sim(kind, n, S, 6)
+    orc = oracle.OracleSim(kind, n, S, 6)
+    acts = inputs.forced_actions(1, T, n, nact)
+    acts[3, :5] = [-3, 7, 100, -128, 2]                   # out-of-range bytes follow the documented rule
+    for t in range(T):
+        nxt, rew, done = sim.step(torch.from_numpy(acts[t]).cuda())
+        o_nxt, o_rew, o_done = orc.step(acts[t])
+        assert_same_bits(to_np(nxt), o_nxt, "next_obs t=%d" % t)
+        assert_same_bits(to_np(rew), o_rew, "rew")
+        assert_same_bits(to_np(done), o_done, "done")
+    ep, rc, tt = sim.counters()
+    assert tt == T and np.array_equal(to_np(rc).astype(np.uint32), orc.reset_count)
+
+
+def test_env_offset_shards_reproduce_the_global_population():
+    torch = torch_cuda()
+    full = oracle.OracleSim(oracle.CARTPOLE, 96, seed=12)
+    ref = full.rollout(50)
+    for off in (0, 32, 64):
+        sim = binding.Sim(oracle.CARTPOLE, 32, 4, 12, env_offset=off)
+        out = sim.rollout(50, 25)
+        for k in ("obs", "act", "done"):
+            assert_same_bits(to_np(out[k]), ref[k][:, off:off + 32], "shard %d %s" % (off, k))
+
+
+def test_checkpoint_resume_and_split_rollout():
+    torch = torch_cuda()
+    a = binding.Sim(oracle.ACROBOT, 130, 4, 2)
+    whole = a.rollout(90, 30)
+    b = binding.Sim(oracle.ACROBOT, 130, 4, 2)
+    first = b.rollout(41, 41)
+    st, (ep, rc, t) = b.state(), b.counters()
+    c = binding.Sim(oracle.ACROBOT, 130, 4, 2)
+    c.set_state(st)
+    c.set_counters(ep, rc, t)
+    second = c.rollout(49, 7)
+    for k in ("obs", "act", "rew", "done"):
+        assert torch.equal(whole[k], torch.cat([first[k], second[k]]))
+    assert torch.equal(a.state(), c.state())
+
+
+def test_null_outputs_and_reset():
+    torch = torch_cuda()
+    sim = binding.Sim(oracle.CARTPOLE, 777, 4, 1)
+    orc = oracle.OracleSim(oracle.CARTPOLE, 777, 4, 1)
+    sim.rollout(33, 33, want=())
+    orc.rollout(33, want=())
+    compare_rollout({}, sim, {}, orc, what="null outputs")
+    only_done = sim.rollout(10, 10, want=("done",))
+    assert only_done["obs"] is None and only_done["done"].shape == (10, 777)
+    sim.reset()
+    orc.reset()
+    compare_rollout({}, sim, {}, orc, what="after reset")
+
+
+def test_rollout_host_matches_device_rollout():
+    torch = torch_cuda()
+    n, T = 513, 37
+    p = inputs.mlp_params(3, 0.1)
+    for params in (None, p):
+        a = binding.Sim(oracle.CARTPOLE, n, 4, 5)
+        dev = a.rollout(T, 8, None if params is None else torch.from_numpy(params).cuda())
+        b = binding.Sim(oracle.CARTPOLE, n, 4, 5)
+        h = {"obs": torch.empty((T, n, 4), dtype=torch.float32).pin_memory(), "act": torch.empty((T, n), dtype=torch.int8).pin_memory(),
+             "rew": torch.empty((T, n), dtype=torch.float32).pin_memory(), "done": torch.empty((T, n), dtype=torch.uint8).pin_memory()}
+        binding.sim_rollout_host(b.h, T, 8, params, h["obs"], h["act"], h["rew"], h["done"])
+        for k in h:
+            assert torch.equal(dev[k].cpu(), h[k]), k
+        assert torch.equal(a.state(), b.state())
+
+
+def test_argument_errors_with_live_handle():
+    torch = torch_cuda()
+    sim = binding.Sim(oracle.ACROBOT, 16)
+    L = binding.lib()
+    assert L.sim_rollout(sim.h, 0, 1, None, None, None, None, None) == binding.SIM_EINVAL
+    assert L.sim_rollout(sim.h, 5, 0, None, None, None, None, None) == binding.SIM_EINVAL
+    p = torch.zeros(4610, device="cuda")
+    assert L.sim_rollout(sim.h, 5, 1, p.data_ptr(), None, None, None, None) == binding.SIM_EINVAL   # MLP is CartPole-only
+    assert L.sim_step(sim.h, None, None, None, None) == binding.SIM_EINVAL
+    assert L.sim_set_env_offset(sim.h, (1 << 32) - 8) == binding.SIM_EINVAL
+    ep, rc, t = sim.counters()
+    assert t == 0                                         # nothing above advanced the handle
