@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the batched environment-stepping hot path on B200.
+
+A "step" is one pass of the whole hot path over one batch: one `sim_rollout` of the workload's
+N envs for its T steps at one K_fused (launch prologue, K x (action selection, physics, reward /
+done, auto-reset, trajectory write), launch epilogue), continuing from the state the previous
+step left.  The metric is environment-steps per second.
+
+    python bench.py                       # cfg2 (CartPole, N=65536, T=1000) at K_fused=1000 + K sweep
+    python bench.py --workload cfg3       # another workload of the table in inputs.py
+    python bench.py --impl reference      # the CPU oracle on the host cores, same metric
+    torchrun ... bench.py --gpus N        # one rank per GPU, disjoint env ranges, no collective in the data path
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2207_07736_b200 import inputs, shard  # noqa: E402
+
+FP32_LANES_PER_SM = 128
+TRAJ_BYTES_S4 = 22          # obs 16 + act 1 + rew 4 + done 1
+# nominal / operation-expanded flops per env-step (fma = 2, any other fp32 op = 1, integer work = 0)
+FLOPS = {"cartpole": (27, 52), "acrobot": (181, 455), "mlp": (9094, 12205)}
+
+
+def algorithmic_bytes_per_env_step(w, K):
+    traj = (4 * w.state_dim + 6) if w.trajectory else 0
+    return traj + (2 * 4 * w.state_dim + 16) / K
+
+
+def nominal_flops_per_env_step(w):
+    if w.env_kind == inputs.SYNTH:
+        return 7 * w.state_dim, 24 * w.state_dim
+    if w.env_kind == inputs.ACROBOT:
+        return FLOPS["acrobot"]
+    base = FLOPS["cartpole"]
+    if w.mlp_seed is not None:
+        return base[0] + FLOPS["mlp"][0], base[1] + FLOPS["mlp"][1]
+    return base
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index, period=0.002):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.max_mhz, self.ok = period, [], set(), None, False
+        self._halt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    NAMES = {0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x4: "sw_power_cap",
+             0x80: "hw_power_brake_slowdown"}
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.NAMES.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=1.0)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_rate(w, budget_s, n_sample=None):
+    """env-steps/s of the single-threaded oracle on a bounded sample of the workload."""
+    import oracle
+    n = n_sample or min(w.n_envs, 256 if w.mlp_seed is not None else max(4, 4096 * 4 // w.state_dim))
+    params = None if w.mlp_seed is None else inputs.mlp_params(w.mlp_seed)
+    ids = inputs.sample_env_ids(3, w.n_envs, n)
+    sim = oracle.OracleSim(w.env_kind, state_dim=w.state_dim, seed=w.seed, env_ids=ids)
+    want = ("obs", "act", "rew", "done") if w.trajectory else ()
+    steps = 0
+    t0 = time.perf_counter()
+    passes = 0
+    while True:
+        sim.rollout(w.T, policy_params=params, want=want)
+        steps += sim.n * w.T
+        passes += 1
+        if time.perf_counter() - t0 >= budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return steps / dt, "%d envs x T=%d x %d passes (%.1f s)" % (sim.n, w.T, passes, dt)
+
+
+def run_reference(args, w):
+    rank, _, world = shard.dist_env()
+    if rank != 0:
+        return 0
+    per_step_budget = max(0.2, min(5.0, 60.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_rate(w, per_step_budget)
+    rates, sample = [], ""
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        r, sample = oracle_rate(w, per_step_budget)
+        rates.append(r)
+    wall = time.perf_counter() - t0
+    v = statistics.mean(rates)
+    line = {
+        "impl": "reference", "metric": "env_steps_per_sec", "value": v, "unit": "env-steps/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "env_kind": w.env_kind, "n_envs": w.n_envs, "T": w.T, "state_dim": w.state_dim},
+        "cpu_baseline": {"value": v, "unit": "env-steps/s", "cores": 1, "kind": "oracle", "sample": "each step: " + sample},
+        "e2e": {"value": v, "unit": "env-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def time_rollouts(torch, sim, w, K, reps, d_params, out):
+    """Device time (ms) of `reps` rollouts, each bracketed by its own pair of events on the sim's stream."""
+    times = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        sim.rollout(w.T, K, d_params, out=out)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return times
+
+
+def run_gpu(args, w):
+    import torch
+    from paper_2207_07736_b200 import binding
+    rank, local_rank, world = shard.dist_env()
+    if world != args.gpus and world > 1:
+        raise SystemExit("--gpus %d but WORLD_SIZE=%d" % (args.gpus, world))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the CPU oracle")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = shard.init_process_group("nccl")
+    hbm_peak, sm_max_mhz, peak_kind = measured_peaks()
+
+    env_offset, n = shard.env_range(rank, world, w.n_envs)
+    K = args.k_fused or max(w.k_sweep)
+    sim = binding.Sim(w.env_kind, n, w.state_dim, w.seed, device=dev, env_offset=env_offset)
+    d_params = None if w.mlp_seed is None else torch.from_numpy(inputs.mlp_params(w.mlp_seed)).to(dev)
+    out = sim.alloc_outputs(w.T) if w.trajectory else {}
+    traj_bytes = sum(t.numel() * t.element_size() for t in out.values() if t is not None)
+
+    def one_step():
+        sim.rollout(w.T, K, d_params, out=out)
+
+    # warm-up: W steps, then keep going until the clocks have had time to ramp (still untimed)
+    for _ in range(args.warmup):
+        one_step()
+    torch.cuda.synchronize()
+    t_ramp = time.perf_counter()
+    while time.perf_counter() - t_ramp < args.ramp_s:
+        one_step()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    launches0 = sim.launches
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        one_step()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    launches = sim.launches - launches0
+    elapsed_ms = e0.elapsed_time(e1)
+    units = float(n) * w.T * args.steps
+    elapsed_ms, units_all = shard.reduce_timing(dist, elapsed_ms, units, device=dev)
+    value = units_all / (elapsed_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel (the fused rollout kernel; ceil(T/K) launches per step)
+    launches_per_step = -(-w.T // K)
+    launch_ms = elapsed_ms / (args.steps * launches_per_step)          # single stream, back-to-back launches
+    bytes_per_env_step = algorithmic_bytes_per_env_step(w, K)
+    k_per_launch = min(K, w.T)
+    bytes_per_launch = bytes_per_env_step * n * k_per_launch
+    fl_nom, fl_exp = nominal_flops_per_env_step(w)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    fp32_peak_tflops = 2 * FP32_LANES_PER_SM * sms * sm_max_mhz * 1e6 / 1e12
+    t_hbm = bytes_per_env_step / (hbm_peak * 1e9)
+    t_alu = fl_nom / (fp32_peak_tflops * 1e12)
+    if t_hbm >= t_alu:
+        achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                    "traffic": args.traffic_bytes, "peak_source": "MEASURED_PEAKS.json (of %s)" % peak_kind,
+                    "algorithmic_bytes_per_launch": bytes_per_launch}
+    else:
+        achieved = fl_nom * n * k_per_launch / (launch_ms * 1e-3) / 1e12
+        roofline = {"bound": "alu", "achieved": achieved, "peak": fp32_peak_tflops, "unit": "TFLOP/s", "frac": achieved / fp32_peak_tflops,
+                    "traffic": args.traffic_bytes, "peak_source": "2 x 128 lanes x %d SMs x %.0f MHz (sm_max_mhz of MEASURED_PEAKS.json, of %s)" % (sms, sm_max_mhz, peak_kind),
+                    "flops_ledger": "nominal %d flop/env-step (operation-expanded: %d)" % (fl_nom, fl_exp),
+                    "frac_expanded_ledger": fl_exp * n * k_per_launch / (launch_ms * 1e-3) / 1e12 / fp32_peak_tflops}
+    roofline["kernel"] = "fused rollout kernel, K_fused=%d, %d launch(es) per step" % (K, launches_per_step)
+    roofline["launch_ms"] = launch_ms
+
+    # ---- K_fused sweep (rank 0 reports its own GPU; same handle, a few repetitions each)
+    sweep = {}
+    if not args.no_sweep:
+        for k in w.k_sweep:
+            reps = max(3, min(args.steps, 10))
+            time_rollouts(torch, sim, w, k, 1, d_params, out)
+            ts = time_rollouts(torch, sim, w, k, reps, d_params, out)
+            med = statistics.median(ts)
+            sweep[str(k)] = {"env_steps_per_sec": n * w.T / (med * 1e-3), "ms": med, "launches": -(-w.T // k),
+                             "bytes_per_env_step": algorithmic_bytes_per_env_step(w, k)}
+        base = sweep.get("1")
+        if base:
+            for k, v in sweep.items():
+                v["fusion_speedup_vs_k1"] = base["ms"] / v["ms"]
+
+    # ---- end to end: host buffers, D2H of the trajectory (and H2D of the policy) inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        if w.trajectory:
+            h = {"obs": torch.empty((w.T, n, w.state_dim), dtype=torch.float32).pin_memory(),
+                 "act": torch.empty((w.T, n), dtype=torch.int8).pin_memory(),
+                 "rew": torch.empty((w.T, n), dtype=torch.float32).pin_memory(),
+                 "done": torch.empty((w.T, n), dtype=torch.uint8).pin_memory()}
+        else:
+            h = {"obs": None, "act": None, "rew": None, "done": torch.empty((w.T, n), dtype=torch.uint8).pin_memory()}
+        h_params = None if w.mlp_seed is None else torch.from_numpy(inputs.mlp_params(w.mlp_seed)).pin_memory()
+        k_host = min(K, max(1, w.T // 8))                               # chunked so that copies overlap compute
+        del out
+        torch.cuda.empty_cache()
+
+        def host_step():
+            binding.sim_rollout_host(sim.h, w.T, k_host, h_params, h["obs"], h["act"], h["rew"], h["done"])
+
+        host_step()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e_steps = max(1, min(args.steps, args.e2e_steps))
+        t0 = time.perf_counter()
+        for _ in range(e_steps):
+            host_step()                                                 # returns after the last copy has landed
+        torch.cuda.synchronize()
+        dt_ms = (time.perf_counter() - t0) * 1e3
+        dt_ms, e_units = shard.reduce_timing(dist, dt_ms, float(n) * w.T * e_steps, device=dev)
+        d2h = sum(t.numel() * t.element_size() for t in h.values() if t is not None)
+        e2e = {"value": e_units / (dt_ms * 1e-3), "unit": "env-steps/s", "h2d_bytes_per_step": 0 if h_params is None else h_params.numel() * 4,
+               "d2h_bytes_per_step": d2h, "steps": e_steps, "k_fused_chunk": k_host,
+               "note": "sim_rollout_host: trajectory copied to pinned host memory chunk by chunk while the next chunk computes"}
+
+    if rank != 0:
+        return 0
+
+    cpu = None
+    if not args.no_cpu and world == 1:
+        v, sample = oracle_rate(w, args.cpu_seconds)
+        cpu = {"value": v, "unit": "env-steps/s", "cores": 1, "kind": "oracle", "sample": sample,
+               "host_cores_available": os.cpu_count()}
+
+    line = {
+        "metric": "env_steps_per_sec", "value": value, "unit": "env-steps/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "env": ["cartpole", "acrobot", "synthetic"][w.env_kind], "n_envs_per_gpu": n, "T": w.T,
+                   "state_dim": w.state_dim, "k_fused": K, "policy": "mlp_4_64_64_2" if w.mlp_seed is not None else "uniform_random",
+                   "trajectory_bytes_per_step": traj_bytes,
+                   "l2": "each step writes %.2f GB of trajectory (> 126 MB L2); no flush between steps" % (traj_bytes / 1e9) if traj_bytes > 2e8
+                   else "state (%.2f GB) streamed from HBM every launch" % (n * w.state_dim * 4 / 1e9),
+                   "parallelism": "dp%d (disjoint env ranges, no collective)" % world},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        "k_sweep": sweep,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--k-fused", type=int, default=0, help="K_fused of the timed steps (default: the largest of the workload's sweep)")
+    ap.add_argument("--ramp-s", type=float, default=0.5, help="extra untimed warm-up so the SM clock ramps before timing")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--traffic-bytes", type=float, default=None, help="ncu dram bytes per launch, if captured for this shape")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    w = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+    return run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
