@@ -31,6 +31,7 @@ SIGNATURES = {
     "sim_get_counters": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_uint64)]),
     "sim_set_counters": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]),
     "sim_policy_logits": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
+    "sim_selfcheck_division": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_uint64)]),
     "sim_launch_count": (C.c_int64, [C.c_void_p]),
     "sim_strerror": (C.c_char_p, [C.c_int]),
     "sim_last_cuda_error": (C.c_int, [C.c_void_p]),
@@ -133,6 +134,12 @@ def sim_set_counters(h, d_ep_len, d_reset_count, t):
 
 def sim_policy_logits(h, d_obs, M, d_params, d_logits):
     _check(lib().sim_policy_logits(h, _ptr(d_obs), M, _ptr(d_params), _ptr(d_logits)), h)
+
+
+def sim_selfcheck_division(h, nums_per_den):
+    out = C.c_uint64()
+    _check(lib().sim_selfcheck_division(h, nums_per_den, C.byref(out)), h)
+    return out.value
 
 
 def sim_launch_count(h):

@@ -169,7 +169,10 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
         a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K;
         a.out_obs = reinterpret_cast<float4 *>(obs); a.out_act = act; a.out_rew = rew; a.out_done = done;
         a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.rk = s->rk;
-        CU(s, launch_s4(s->env_kind, policy, a, s->stream));
+        if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM)
+            CU(s, launch_cartpole_random(a, s->stream));
+        else
+            CU(s, launch_s4(s->env_kind, policy, a, s->stream));
     }
     s->launches += 1;
     s->t += (uint64_t)K;
@@ -314,5 +317,22 @@ SIM_API int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const flo
     if (!s || !d_obs || !d_params || !d_logits || M < 0) return SIM_EINVAL;
     CU(s, launch_policy_logits(d_obs, M, d_params, d_logits, s->stream));
     if (M > 0) s->launches += 1;
+    return SIM_OK;
+}
+
+SIM_API int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_mismatches)
+{
+    if (!s || !h_mismatches || nums_per_den < 0) return SIM_EINVAL;
+    unsigned long long *d_bad = nullptr;
+    CU(s, cudaMalloc(&d_bad, sizeof(unsigned long long)));
+    cudaError_t e = cudaMemsetAsync(d_bad, 0, sizeof(unsigned long long), s->stream);
+    if (e == cudaSuccess) e = launch_division_selfcheck(nums_per_den, d_bad, s->stream);
+    unsigned long long h = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&h, d_bad, sizeof(h), cudaMemcpyDeviceToHost, s->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+    cudaFree(d_bad);
+    if (e != cudaSuccess) return cuda_fail(s, e);
+    s->launches += 1;
+    *h_mismatches = (uint64_t)h;
     return SIM_OK;
 }

@@ -183,6 +183,33 @@ def test_rollout_host_matches_device_rollout():
         assert torch.equal(a.state(), b.state())
 
 
+def test_fused_cartpole_division_is_ieee_on_this_device():
+    torch_cuda()
+    sim = binding.Sim(oracle.CARTPOLE, 8)
+    # every possible denominator x 2048 numerators (1.7e9 quotients) and every reciprocal
+    assert binding.sim_selfcheck_division(sim.h, 2048) == 0
+
+
+def test_cartpole_window_path_edge_cases():
+    """States the straight-line window cannot promise anything about: angles far outside 12 degrees
+    (general sin/cos), huge velocities (numerator outside the guarded range, infinities), states that
+    terminate at once and repeatedly, exact zeros.  All must replay through the plain path and match."""
+    def pre(sim, orc, torch):
+        rng = np.random.default_rng(5)
+        st = orc.state.copy()
+        st[0::7] = (rng.uniform(-1, 1, st[0::7].shape) * np.array([2.3, 2.0, 3.0, 2.0])).astype(np.float32)   # |theta| up to 3 rad
+        st[1::7, 3] = 1e18                       # theta_dot^2 overflows
+        st[2::7, 2] = 0.2094                     # one step from the limit
+        st[3::7] = 0.0                           # exact zeros: numerator of the division is +-10/1.1 * 1, fine; theta = 0
+        st[4::7, 1] = 1e-30                      # tiny velocities
+        st[5::7, 0] = 2.3999
+        st[5::7, 1] = 3.0
+        orc.state[:] = st
+        sim.set_state(torch.from_numpy(st).cuda())
+    for K in (1, 8, 16, 40):
+        run_pair(oracle.CARTPOLE, 515, 40, K, seed=21, pre=pre)
+
+
 def test_argument_errors_with_live_handle():
     torch = torch_cuda()
     sim = binding.Sim(oracle.ACROBOT, 16)
