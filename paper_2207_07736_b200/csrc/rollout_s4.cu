@@ -1,4 +1,5 @@
-// Fused multi-step rollout for envs with a 4-float state (CartPole, Acrobot): one thread owns
+// Generic fused multi-step rollout for envs with a 4-float state (Acrobot; CartPole with caller-given
+// actions): one thread owns
 // one env, keeps its state and counters in registers for the K steps of the launch, and streams
 // the per-step trajectory rows to global memory with coalesced stores (obs as one float4 per
 // env, so a warp writes 512 contiguous bytes).
@@ -6,92 +7,6 @@
 #include "sim_envs.cuh"
 
 namespace simk {
-
-// ---------------------------------------------------------------------------------------------
-// MLP policy 4 -> 64 -> 64 -> 2 (tanh).  The parameters are staged once per CTA into shared
-// memory, layer 2 transposed so that the weights of consecutive output units for one input are
-// contiguous (one 128-bit broadcast load feeds four accumulators).  Every output unit is one
-// sequential fma chain over its inputs in ascending order, starting from the bias.
-// ---------------------------------------------------------------------------------------------
-struct MlpSmem {
-    float4 w1[64];        // w1[j] = W1[j][0..3]
-    float b1[64];
-    float w2t[64 * 64];   // w2t[k*64 + j] = W2[j][k]
-    float b2[64];
-    float2 w3[64];        // w3[j] = (W3[0][j], W3[1][j])
-    float b3[2];
-};
-
-__device__ __forceinline__ void stage_mlp(const float *__restrict__ p, MlpSmem &s)
-{
-    const int tid = threadIdx.x, nt = blockDim.x;
-    for (int i = tid; i < 64; i += nt) {
-        s.w1[i] = make_float4(p[i * 4 + 0], p[i * 4 + 1], p[i * 4 + 2], p[i * 4 + 3]);
-        s.b1[i] = p[256 + i];
-        s.b2[i] = p[4416 + i];
-        s.w3[i] = make_float2(p[4480 + i], p[4544 + i]);
-    }
-    for (int i = tid; i < 4096; i += nt) {
-        const int j = i >> 6, k = i & 63;              // coalesced read of W2[j][k]
-        s.w2t[k * 64 + j] = p[320 + i];
-    }
-    if (tid < 2) s.b3[tid] = p[4608 + tid];
-    __syncthreads();
-}
-
-__device__ __forceinline__ void mlp_logits(const float4 obs, const MlpSmem &s, float &l0, float &l1)
-{
-    float h1[64];
-#pragma unroll
-    for (int j = 0; j < 64; ++j) {
-        const float4 w = s.w1[j];
-        float acc = s.b1[j];
-        acc = __fmaf_rn(w.x, obs.x, acc);
-        acc = __fmaf_rn(w.y, obs.y, acc);
-        acc = __fmaf_rn(w.z, obs.z, acc);
-        acc = __fmaf_rn(w.w, obs.w, acc);
-        h1[j] = tanh_s(acc);
-    }
-    l0 = s.b3[0];
-    l1 = s.b3[1];
-#pragma unroll 1
-    for (int jb = 0; jb < 64; jb += 8) {
-        float acc[8];
-        {
-            const float4 ba = *reinterpret_cast<const float4 *>(&s.b2[jb]);
-            const float4 bb = *reinterpret_cast<const float4 *>(&s.b2[jb + 4]);
-            acc[0] = ba.x; acc[1] = ba.y; acc[2] = ba.z; acc[3] = ba.w;
-            acc[4] = bb.x; acc[5] = bb.y; acc[6] = bb.z; acc[7] = bb.w;
-        }
-#pragma unroll
-        for (int k = 0; k < 64; ++k) {
-            const float4 wa = *reinterpret_cast<const float4 *>(&s.w2t[k * 64 + jb]);
-            const float4 wb = *reinterpret_cast<const float4 *>(&s.w2t[k * 64 + jb + 4]);
-            const float h = h1[k];
-            acc[0] = __fmaf_rn(wa.x, h, acc[0]); acc[1] = __fmaf_rn(wa.y, h, acc[1]);
-            acc[2] = __fmaf_rn(wa.z, h, acc[2]); acc[3] = __fmaf_rn(wa.w, h, acc[3]);
-            acc[4] = __fmaf_rn(wb.x, h, acc[4]); acc[5] = __fmaf_rn(wb.y, h, acc[5]);
-            acc[6] = __fmaf_rn(wb.z, h, acc[6]); acc[7] = __fmaf_rn(wb.w, h, acc[7]);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float h2 = tanh_s(acc[i]);
-            const float2 w3 = s.w3[jb + i];
-            l0 = __fmaf_rn(w3.x, h2, l0);
-            l1 = __fmaf_rn(w3.y, h2, l1);
-        }
-    }
-}
-
-// Inverse-CDF sample over the two unnormalised softmax weights: action 0 iff u*(e0+e1) < e0.
-__device__ __forceinline__ int sample2(float l0, float l1, uint32_t w)
-{
-    const float m = fmaxf(l0, l1);
-    const float e0 = exp_s(__fsub_rn(l0, m));
-    const float e1 = exp_s(__fsub_rn(l1, m));
-    const float thr = __fmul_rn(uniform01(w), __fadd_rn(e0, e1));
-    return (thr < e0) ? 0 : 1;
-}
 
 // ---------------------------------------------------------------------------------------------
 // The rollout kernel.
@@ -120,17 +35,12 @@ __device__ __forceinline__ bool env_step(float4 &s, int &act, uint32_t &len, flo
     }
 }
 
-constexpr int kS4Threads = 64;      // small CTAs spread 65 536 envs evenly over 148 SMs
-constexpr int kMlpThreads = 128;
+constexpr int kS4Threads = 64;      // small CTAs spread the envs evenly over 148 SMs
 
 template <int ENV, int POLICY>
-__global__ void __launch_bounds__(POLICY == POLICY_MLP ? kMlpThreads : kS4Threads)
+__global__ void __launch_bounds__(kS4Threads)
 rollout_s4_kernel(const __grid_constant__ S4Args a)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    MlpSmem &ms = *reinterpret_cast<MlpSmem *>(smem_raw);
-    if (POLICY == POLICY_MLP) stage_mlp(a.params, ms);
-
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= a.n) return;
     const uint32_t env = a.env_offset + i;
@@ -155,10 +65,6 @@ rollout_s4_kernel(const __grid_constant__ S4Args a)
             int act;
             if (POLICY == POLICY_GIVEN) {
                 act = a.actions[i];
-            } else if (POLICY == POLICY_MLP) {
-                float l0, l1;
-                mlp_logits(s, ms, l0, l1);
-                act = sample2(l0, l1, w);
             } else {
                 act = random_action<ENV>(w);
             }
@@ -210,19 +116,6 @@ reset_synth_kernel(float4 *state, uint32_t *ep_len, uint32_t *reset_count, uint3
     if (j == 0) { ep_len[i] = 0u; reset_count[i] = 0u; }
 }
 
-__global__ void __launch_bounds__(kMlpThreads)
-policy_logits_kernel(const float4 *__restrict__ obs, int64_t M, const float *__restrict__ params, float2 *__restrict__ logits)
-{
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    MlpSmem &ms = *reinterpret_cast<MlpSmem *>(smem_raw);
-    stage_mlp(params, ms);
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= M) return;
-    float l0, l1;
-    mlp_logits(obs[i], ms, l0, l1);
-    logits[i] = make_float2(l0, l1);
-}
-
 // ---------------------------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------------------------
@@ -249,10 +142,8 @@ cudaError_t launch_reset(int env_kind, int S, float *state, uint32_t *ep_len, ui
 template <int ENV, int POLICY>
 static cudaError_t launch_s4_t(const S4Args &a, cudaStream_t st)
 {
-    constexpr int threads = POLICY == POLICY_MLP ? kMlpThreads : kS4Threads;
-    const size_t smem = POLICY == POLICY_MLP ? sizeof(MlpSmem) : 0;
-    const unsigned blocks = (a.n + threads - 1u) / threads;
-    rollout_s4_kernel<ENV, POLICY><<<blocks, threads, smem, st>>>(a);
+    const unsigned blocks = (a.n + kS4Threads - 1u) / kS4Threads;
+    rollout_s4_kernel<ENV, POLICY><<<blocks, kS4Threads, 0, st>>>(a);
     return cudaGetLastError();
 }
 
@@ -261,22 +152,11 @@ cudaError_t launch_s4(int env_kind, int policy, const S4Args &a, cudaStream_t st
     if (env_kind == ENV_CARTPOLE) {
         if (policy == POLICY_RANDOM) return launch_s4_t<ENV_CARTPOLE, POLICY_RANDOM>(a, st);
         if (policy == POLICY_GIVEN) return launch_s4_t<ENV_CARTPOLE, POLICY_GIVEN>(a, st);
-        if (policy == POLICY_MLP) return launch_s4_t<ENV_CARTPOLE, POLICY_MLP>(a, st);
     } else if (env_kind == ENV_ACROBOT) {
         if (policy == POLICY_RANDOM) return launch_s4_t<ENV_ACROBOT, POLICY_RANDOM>(a, st);
         if (policy == POLICY_GIVEN) return launch_s4_t<ENV_ACROBOT, POLICY_GIVEN>(a, st);
     }
     return cudaErrorInvalidValue;
-}
-
-cudaError_t launch_policy_logits(const float *obs, int64_t M, const float *params, float *logits, cudaStream_t st)
-{
-    if (M <= 0) return cudaSuccess;
-    const int64_t blocks = (M + kMlpThreads - 1) / kMlpThreads;
-    if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
-    policy_logits_kernel<<<(unsigned)blocks, kMlpThreads, sizeof(MlpSmem), st>>>(reinterpret_cast<const float4 *>(obs), M, params,
-                                                                                reinterpret_cast<float2 *>(logits));
-    return cudaGetLastError();
 }
 
 }  // namespace simk

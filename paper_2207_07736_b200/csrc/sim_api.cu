@@ -171,6 +171,8 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
         a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.rk = s->rk;
         if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM)
             CU(s, launch_cartpole_random(a, s->stream));
+        else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP)
+            CU(s, launch_cartpole_mlp(a, s->stream));
         else
             CU(s, launch_s4(s->env_kind, policy, a, s->stream));
     }

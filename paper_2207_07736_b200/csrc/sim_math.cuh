@@ -174,4 +174,46 @@ __device__ __forceinline__ void sincos2(f2 x, f2 &sn, f2 &cs, uint32_t converged
     }
 }
 
+__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
+// exp of two arguments already inside [-87, 88] (same operations as exp_core, two at a time).
+__device__ __forceinline__ f2 exp2_core(f2 y)
+{
+    const f2 magic = splat(kRoundMagic);
+    const f2 t = mul2(y, splat(fbits(0x3FB8AA3Bu)));
+    const f2 nb = add2(t, magic);
+    const f2 nn = sub2(magic, nb);
+    f2 r = fma2(nn, splat(fbits(0x3F317218u)), y);
+    r = fma2(nn, splat(fbits(0xB102E308u)), r);
+    f2 p = fma2(splat(fbits(0x39500D01u)), r, splat(fbits(0x3AB60B61u)));
+    p = fma2(p, r, splat(fbits(0x3C088889u)));
+    p = fma2(p, r, splat(fbits(0x3D2AAAABu)));
+    p = fma2(p, r, splat(fbits(0x3E2AAAABu)));
+    p = fma2(p, r, splat(0.5f));
+    p = fma2(p, r, splat(1.0f));
+    p = fma2(p, r, splat(1.0f));
+    const f2 scale = pk(__uint_as_float((__float_as_uint(lo(nb)) << 23) + 0x3F800000u),
+                        __uint_as_float((__float_as_uint(hi(nb)) << 23) + 0x3F800000u));
+    return mul2(p, scale);
+}
+
+// tanh of two arguments.  d = exp(2|x|) + 1 lies in [2, 2^27) whenever the result is used, where one
+// Newton step from the hardware reciprocal is the correctly rounded reciprocal (checked exhaustively
+// on the device by the library's arithmetic self-check), so 1 - 2/d is one more fused multiply-add.
+__device__ __forceinline__ f2 tanh2(f2 x)
+{
+    const float xa = lo(x), xb = hi(x);
+    const float aa = fabsf(xa), ab = fabsf(xb);
+    const f2 a = pk(aa, ab);
+    const f2 e = exp2_core(add2(a, a));
+    const f2 d = add2(e, splat(1.0f));
+    const f2 nd = fma2(e, splat(-1.0f), splat(-1.0f));            // -d exactly
+    const f2 y0 = pk(rcp_approx(lo(d)), rcp_approx(hi(d)));
+    const f2 y1 = fma2(y0, fma2(nd, y0, splat(1.0f)), y0);
+    const f2 t = fma2(splat(-2.0f), y1, splat(1.0f));
+    const float ta = aa > 9.0f ? 1.0f : lo(t);
+    const float tb = ab > 9.0f ? 1.0f : hi(t);
+    return pk(copysignf(ta, xa), copysignf(tb, xb));
+}
+
 }  // namespace simk
