@@ -344,6 +344,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--traffic-bytes", type=float, default=None, help="ncu dram bytes per launch, if captured for this shape")
+    ap.add_argument("--n-envs", type=int, default=0, help="override the workload's env count (profiling on a reduced case)")
+    ap.add_argument("--T", type=int, default=0, help="override the workload's step count (profiling on a reduced case)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -351,6 +353,9 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     w = inputs.WORKLOADS[args.workload]
+    if args.n_envs or args.T:
+        import dataclasses
+        w = dataclasses.replace(w, name=w.name + "_reduced", n_envs=args.n_envs or w.n_envs, T=args.T or w.T)
     if args.impl == "reference":
         return run_reference(args, w)
     return run_gpu(args, w)
