@@ -40,7 +40,7 @@ extern "C" {
 typedef struct sim sim_t;   /* opaque */
 
 enum { SIM_CARTPOLE = 0, SIM_ACROBOT = 1, SIM_SYNTH = 2 };
-enum { SIM_OK = 0, SIM_EINVAL = -1, SIM_ENOMEM = -2, SIM_ECUDA = -3, SIM_ESTATE = -4 };
+enum { SIM_OK = 0, SIM_EINVAL = -1, SIM_ENOMEM = -2, SIM_ECUDA = -3, SIM_ESTATE = -4, SIM_ECAPACITY = -5 };
 
 #define SIM_POLICY_PARAM_COUNT 4610   /* W1[64][4] b1[64] W2[64][64] b2[64] W3[2][64] b3[2], rows = output units */
 
@@ -132,6 +132,39 @@ int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_pa
  * guarded exponent range.  *h_mismatches (host) = reciprocal mismatches * 2^32 + quotient
  * mismatches; 0 means the kernel's division is the IEEE division on this device.  Synchronises. */
 int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_mismatches);
+
+/*
+ * sim_rollout_noalloc -- reset N envs and roll them out for T steps without allocating anything
+ * (the paper has no counterpart: it is an addition for callers that cannot allocate).
+ *
+ * Who needs it: a latency-critical loop that must not call cudaMalloc / cudaFree because both
+ * stall every stream of the device; a process whose device memory has been handed out in full to
+ * another allocator; a component that may only touch the buffers it is given.  Instead of the
+ * buffers sim_create would allocate, the per-env working memory (state matrix, episode lengths,
+ * reset counts) sits in a fixed array of SIM_NOALLOC_SCRATCH_BYTES inside the library's device
+ * image; every GPU that loads the library holds that array until the process exits.
+ *
+ *   env_kind, n_envs, state_dim, seed   as in sim_create; env offset 0.
+ *   T, K_fused, d_policy_params, out_*  as in sim_rollout (device pointers, outputs nullable);
+ *                                       the rollout starts from the freshly drawn state at t = 0,
+ *                                       so the outputs equal sim_create + sim_rollout bit for bit.
+ *   cuda_stream                         cudaStream_t as void*, NULL = default stream.  Work is
+ *                                       only enqueued; the caller synchronises.
+ * Limit: 256-aligned(4*state_dim*n_envs) + 2 * 256-aligned(4*n_envs) bytes must not exceed
+ * SIM_NOALLOC_SCRATCH_BYTES (e.g. 349 440 four-float envs); larger problems return
+ * SIM_ECAPACITY and enqueue nothing.  Other errors: SIM_EINVAL, SIM_ECUDA.
+ * The call makes no cudaMalloc, cudaFree or other allocating call, on the host or the device.
+ * First use on a device looks up the array's device address (once per device, with that device
+ * current): make that first call outside any stream capture.
+ * All calls share the one array.  It keeps the previous call's contents; each call rewrites every
+ * word it later reads before reading it, so nothing needs clearing by the caller -- but two
+ * calls whose work overlaps on the GPU (different streams, or one process-wide device shared by
+ * threads) race on it and corrupt each other.  Serialise them.
+ */
+#define SIM_NOALLOC_SCRATCH_BYTES (8u << 20)
+int sim_rollout_noalloc(int env_kind, int64_t n_envs, int state_dim, uint64_t seed, int T, int K_fused,
+                        const float *d_policy_params, float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done,
+                        void *cuda_stream);
 
 /* sim_launch_count -- kernels launched by this handle since creation (for launch accounting). */
 int64_t sim_launch_count(sim_t *s);

@@ -13,7 +13,8 @@ _HERE = Path(__file__).resolve().parent
 LIB_PATH = _HERE / "libsim_b200.so"
 
 SIM_CARTPOLE, SIM_ACROBOT, SIM_SYNTH = 0, 1, 2
-SIM_OK, SIM_EINVAL, SIM_ENOMEM, SIM_ECUDA, SIM_ESTATE = 0, -1, -2, -3, -4
+SIM_OK, SIM_EINVAL, SIM_ENOMEM, SIM_ECUDA, SIM_ESTATE, SIM_ECAPACITY = 0, -1, -2, -3, -4, -5
+SIM_NOALLOC_SCRATCH_BYTES = 8 << 20
 SIM_POLICY_PARAM_COUNT = 4610
 
 # name -> (restype, argtypes); one entry per declaration in include/sim.h
@@ -32,6 +33,8 @@ SIGNATURES = {
     "sim_set_counters": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]),
     "sim_policy_logits": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "sim_selfcheck_division": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_uint64)]),
+    "sim_rollout_noalloc": (C.c_int, [C.c_int, C.c_int64, C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_void_p, C.c_void_p]),
     "sim_launch_count": (C.c_int64, [C.c_void_p]),
     "sim_strerror": (C.c_char_p, [C.c_int]),
     "sim_last_cuda_error": (C.c_int, [C.c_void_p]),
@@ -140,6 +143,13 @@ def sim_selfcheck_division(h, nums_per_den):
     out = C.c_uint64()
     _check(lib().sim_selfcheck_division(h, nums_per_den, C.byref(out)), h)
     return out.value
+
+
+def sim_rollout_noalloc(env_kind, n_envs, state_dim, seed, T, K_fused, d_policy_params=None, out_obs=None, out_act=None,
+                        out_rew=None, out_done=None, cuda_stream=None):
+    """Reset + rollout using the library's fixed scratch array; allocates nothing (see include/sim.h)."""
+    _check(lib().sim_rollout_noalloc(env_kind, n_envs, state_dim, seed, T, K_fused, _ptr(d_policy_params), _ptr(out_obs), _ptr(out_act),
+                                     _ptr(out_rew), _ptr(out_done), C.c_void_p(cuda_stream) if cuda_stream else None))
 
 
 def sim_launch_count(h):

@@ -66,6 +66,7 @@ SIM_API const char *sim_strerror(int code)
     case SIM_ENOMEM: return "out of device memory";
     case SIM_ECUDA: return "CUDA error (see sim_last_cuda_error)";
     case SIM_ESTATE: return "call not valid in the handle's current state";
+    case SIM_ECAPACITY: return "problem does not fit the fixed scratch array of the no-allocation entry point";
     default: return "unknown error code";
     }
 }
