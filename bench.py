@@ -31,6 +31,9 @@ FP32_LANES_PER_SM = 128
 TRAJ_BYTES_S4 = 22          # obs 16 + act 1 + rew 4 + done 1
 # nominal / operation-expanded flops per env-step (fma = 2, any other fp32 op = 1, integer work = 0)
 FLOPS = {"cartpole": (27, 52), "acrobot": (181, 455), "mlp": (9094, 12205)}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused rollout kernel, from the ncu
+# captures summarised under profiles/ (keyed by workload and K_fused; other shapes report null)
+NCU_TRAFFIC_BYTES = {("cfg2", 1000): 1.3869e9}
 
 
 def algorithmic_bytes_per_env_step(w, K):
@@ -254,6 +257,8 @@ def run_gpu(args, w):
                     "traffic": args.traffic_bytes, "peak_source": "2 x 128 lanes x %d SMs x %.0f MHz (sm_max_mhz of MEASURED_PEAKS.json, of %s)" % (sms, sm_max_mhz, peak_kind),
                     "flops_ledger": "nominal %d flop/env-step (operation-expanded: %d)" % (fl_nom, fl_exp),
                     "frac_expanded_ledger": fl_exp * n * k_per_launch / (launch_ms * 1e-3) / 1e12 / fp32_peak_tflops}
+    if roofline["traffic"] is None:
+        roofline["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, K))
     roofline["kernel"] = "fused rollout kernel, K_fused=%d, %d launch(es) per step" % (K, launches_per_step)
     roofline["launch_ms"] = launch_ms
 
