@@ -1,12 +1,15 @@
 // Fused multi-step rollout of the synthetic S-float simulator (the "state factor" experiment:
 // S times the state, S times the global loads and stores per unfused step).
 //
-// Mapping: an env's S floats are split into L = S/E contiguous chunks of E floats, one chunk
-// per thread, held in registers for all K steps of the launch.  L <= 32: the L threads of an env
-// are adjacent lanes of one warp (several envs per warp when L < 32) and exchange the one halo
-// element and the partial sums with shuffles.  L > 32: one CTA per env, the warps exchange
-// through shared memory.  The sum of squares follows an adjacent-pairs-first binary tree over
-// the element index: inside a chunk, then across lanes by xor-shuffles, then across warps.
+// Mapping: an env's S floats are split into L = S/E contiguous chunks of E floats, one chunk per
+// thread, held in registers for all K steps of the launch.  L <= 32: the L threads of an env are
+// adjacent lanes of one warp (several envs per warp when L < 32) and exchange the one halo element
+// and the partial sums with shuffles.  L > 32: one CTA per env, the warps exchange through shared
+// memory.  Inside a chunk, element j travels with element j + E/2 as one packed fp32 pair, so the
+// "right neighbour" operand of pair j is simply pair j+1 and one issue slot updates two elements.
+// The sum of squares follows an adjacent-pairs-first binary tree over the element index: inside
+// each half chunk (both halves at once, packed), the two halves, then lanes by xor-shuffles, then
+// warps.
 #include "sim_internal.h"
 #include "sim_envs.cuh"
 
@@ -14,41 +17,56 @@ namespace simk {
 
 template <int S> struct SynthShape {
     static constexpr int E = S <= 128 ? 4 : (S <= 512 ? S / 32 : 16);   // floats per thread
+    static constexpr int H = E / 2;                                     // packed pairs per thread
     static constexpr int L = S / E;                                     // threads per env
     static constexpr int WARPS = L > 32 ? L / 32 : 1;                   // warps per env when L > 32
     static constexpr int THREADS = L > 32 ? L : 256;
-    static constexpr int ENVS_PER_CTA = THREADS / L;
+    static constexpr int ENVS_PER_CTA = THREADS / L;                    // envs per tile
 };
 
+// sin of two arguments (general quadrant): both polynomials packed, then one select and one sign
+// flip per element.
+__device__ __forceinline__ f2 sin2(f2 x)
+{
+    const f2 magic = splat(kRoundMagic);
+    const f2 t = mul2(x, splat(fbits(0x3F22F983u)));
+    const f2 nb = add2(t, magic);
+    const f2 nk = sub2(magic, nb);
+    f2 r = fma2(nk, splat(fbits(0x3FC90FDBu)), x);
+    r = fma2(nk, splat(fbits(0xB33BBD2Eu)), r);
+    r = fma2(nk, splat(fbits(0xA6F72CEDu)), r);
+    const f2 r2 = mul2(r, r);
+    f2 p = fma2(splat(fbits(0x3638EF1Du)), r2, splat(fbits(0xB9500D01u)));
+    p = fma2(p, r2, splat(fbits(0x3C088889u)));
+    p = fma2(p, r2, splat(fbits(0xBE2AAAABu)));
+    const f2 Sv = fma2(p, mul2(r2, r), r);
+    f2 c = fma2(splat(fbits(0xB493F27Eu)), r2, splat(fbits(0x37D00D01u)));
+    c = fma2(c, r2, splat(fbits(0xBAB60B61u)));
+    c = fma2(c, r2, splat(fbits(0x3D2AAAABu)));
+    c = fma2(c, r2, splat(-0.5f));
+    const f2 Cv = fma2(c, r2, splat(1.0f));
+    const uint32_t qa = __float_as_uint(lo(nb)), qb = __float_as_uint(hi(nb));
+    const float sa = (qa & 1u) ? lo(Cv) : lo(Sv);
+    const float sb = (qb & 1u) ? hi(Cv) : hi(Sv);
+    return pk(__uint_as_float(__float_as_uint(sa) ^ ((qa << 30) & 0x80000000u)),
+              __uint_as_float(__float_as_uint(sb) ^ ((qb << 30) & 0x80000000u)));
+}
+
+// Shared memory used for the cross-warp exchange of one env (L > 32).
+template <int W> struct SynthExchange { float halo[W]; float sum[W]; };
+
+// K steps of one chunk held in registers.  P[j] = (x_j, x_{j+H}).  All threads of a CTA call this
+// together (it contains CTA barriers when an env spans several warps).
 template <int S>
-__global__ void __launch_bounds__(SynthShape<S>::THREADS)
-rollout_synth_kernel(const __grid_constant__ SynthArgs a)
+__device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[SynthShape<S>::H], uint32_t &len, uint32_t &rc,
+                                            uint32_t i, bool valid, uint32_t sub, SynthExchange<SynthShape<S>::WARPS> &xc)
 {
     using Sh = SynthShape<S>;
-    constexpr int E = Sh::E, L = Sh::L, W = Sh::WARPS;
+    constexpr int E = Sh::E, H = Sh::H, L = Sh::L, W = Sh::WARPS;
     constexpr int LS = L < 32 ? L : 32;                 // lanes of one env inside a warp
-    __shared__ float sm_halo[W];
-    __shared__ float sm_sum[W];
-
-    const uint32_t tid = threadIdx.x;
-    const uint32_t lane = tid & 31u;
-    const uint32_t warp = tid >> 5;
-    const uint32_t sub = tid % L;                       // this thread's chunk index inside its env
-    uint32_t i = blockIdx.x * (uint32_t)Sh::ENVS_PER_CTA + tid / L;
-    const bool valid = i < a.n;                         // tail threads compute on env n-1 and store nothing
-    if (!valid) i = a.n - 1u;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t env = a.env_offset + i;
     const bool leader = valid && sub == 0;
-
-    float x[E];
-    const float *src = a.state + (size_t)i * S + (size_t)sub * E;
-#pragma unroll
-    for (int v = 0; v < E / 4; ++v) {
-        const float4 f = *reinterpret_cast<const float4 *>(src + 4 * v);
-        x[4 * v + 0] = f.x; x[4 * v + 1] = f.y; x[4 * v + 2] = f.z; x[4 * v + 3] = f.w;
-    }
-    uint32_t len = a.ep_len[i];
-    uint32_t rc = a.reset_count[i];
     size_t row = i;
 
     const int nblk = (a.phase + a.K + 3) >> 2;
@@ -56,60 +74,67 @@ rollout_synth_kernel(const __grid_constant__ SynthArgs a)
         uint4 blk = make_uint4(0u, 0u, 0u, 0u);
         if (!a.actions) blk = philox(env, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
 #pragma unroll 1
-        for (int j = 0; j < 4; ++j) {
-            const int k = 4 * b + j - a.phase;
+        for (int j4 = 0; j4 < 4; ++j4) {
+            const int k = 4 * b + j4 - a.phase;
             if (k < 0 || k >= a.K) continue;
-            const uint32_t w = j == 0 ? blk.x : j == 1 ? blk.y : j == 2 ? blk.z : blk.w;
+            const uint32_t w = j4 == 0 ? blk.x : j4 == 1 ? blk.y : j4 == 2 ? blk.z : blk.w;
 
             if (a.out_obs && valid) {
                 float *dst = a.out_obs + row * S + (size_t)sub * E;
+                float xo[E];
+#pragma unroll
+                for (int j = 0; j < H; ++j) { xo[j] = lo(P[j]); xo[j + H] = hi(P[j]); }
 #pragma unroll
                 for (int v = 0; v < E / 4; ++v)
-                    __stcs(reinterpret_cast<float4 *>(dst + 4 * v), make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]));
+                    __stcs(reinterpret_cast<float4 *>(dst + 4 * v), make_float4(xo[4 * v], xo[4 * v + 1], xo[4 * v + 2], xo[4 * v + 3]));
             }
 
             const int act = a.actions ? (a.actions[i] != 0) : (int)(w >> 31);
-            const float c = __fmul_rn(fbits(0x3A83126Fu), act ? 1.0f : -1.0f);
+            const f2 c = splat(__fmul_rn(fbits(0x3A83126Fu), act ? 1.0f : -1.0f));
 
             // halo: first element of the next chunk of the same env (wrapping around)
+            const float x0 = lo(P[0]);
             float halo;
             if (L == 1) {
-                halo = x[0];
+                halo = x0;
             } else {
-                halo = __shfl_sync(0xFFFFFFFFu, x[0], (lane & ~(uint32_t)(LS - 1)) | ((lane + 1u) & (uint32_t)(LS - 1)));
+                halo = __shfl_sync(0xFFFFFFFFu, x0, (lane & ~(uint32_t)(LS - 1)) | ((lane + 1u) & (uint32_t)(LS - 1)));
                 if (W > 1) {
-                    if (lane == 0) sm_halo[warp] = x[0];
+                    if (lane == 0) xc.halo[warp] = x0;
                     __syncthreads();
-                    if (lane == 31) halo = sm_halo[(warp + 1u) % W];
+                    if (lane == 31) halo = xc.halo[(warp + 1u) % W];
                 }
             }
 
-            // Jacobi update: every right-hand side reads pre-step values
-            float q[E];
+            // Jacobi update: every right-hand side reads pre-step values.  The right neighbours of
+            // pair j = (x_j, x_{j+H}) are pair j+1; the last pair's are (x_H, halo).
+            const f2 wrap = pk(hi(P[0]), halo);
+            const f2 c01 = splat(fbits(0x3C23D70Au));
+            f2 Q[H];
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const float right = e + 1 < E ? x[e + 1] : halo;
-                const float z = sin_s(__fadd_rn(x[e], right));
-                q[e] = __fadd_rn(__fmaf_rn(fbits(0x3C23D70Au), z, x[e]), c);
+            for (int j = 0; j < H; ++j) {
+                const f2 right = j + 1 < H ? P[j + 1] : wrap;
+                const f2 z = sin2(add2(P[j], right));
+                Q[j] = add2(fma2(c01, z, P[j]), c);
             }
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                x[e] = q[e];
-                q[e] = __fmul_rn(q[e], q[e]);
+            for (int j = 0; j < H; ++j) {
+                P[j] = Q[j];
+                Q[j] = mul2(Q[j], Q[j]);
             }
 #pragma unroll
-            for (int wdt = 1; wdt < E; wdt <<= 1)
+            for (int wdt = 1; wdt < H; wdt <<= 1)
 #pragma unroll
-                for (int e = 0; e < E; e += 2 * wdt) q[e] = __fadd_rn(q[e], q[e + wdt]);
-            float sum = q[0];
+                for (int j = 0; j < H; j += 2 * wdt) Q[j] = add2(Q[j], Q[j + wdt]);
+            float sum = __fadd_rn(lo(Q[0]), hi(Q[0]));               // left half + right half of the chunk
 #pragma unroll
             for (int m = 1; m < LS; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
             if (W > 1) {
-                if (lane == 0) sm_sum[warp] = sum;
+                if (lane == 0) xc.sum[warp] = sum;
                 __syncthreads();
                 float part[W];
 #pragma unroll
-                for (int v = 0; v < W; ++v) part[v] = sm_sum[v];
+                for (int v = 0; v < W; ++v) part[v] = xc.sum[v];
 #pragma unroll
                 for (int wdt = 1; wdt < W; wdt <<= 1)
 #pragma unroll
@@ -127,38 +152,76 @@ rollout_synth_kernel(const __grid_constant__ SynthArgs a)
 
             if (done) {                                     // uniform over the threads of one env
                 rc += 1u;
+                float xr[E];
 #pragma unroll
                 for (int v = 0; v < E / 4; ++v) {
                     const float4 f = draw_state4<ENV_SYNTH>(env, rc, sub * (uint32_t)(E / 4) + (uint32_t)v, a.rk);
-                    x[4 * v + 0] = f.x; x[4 * v + 1] = f.y; x[4 * v + 2] = f.z; x[4 * v + 3] = f.w;
+                    xr[4 * v + 0] = f.x; xr[4 * v + 1] = f.y; xr[4 * v + 2] = f.z; xr[4 * v + 3] = f.w;
                 }
+#pragma unroll
+                for (int j = 0; j < H; ++j) P[j] = pk(xr[j], xr[j + H]);
                 len = 0u;
             }
             row += a.n;
         }
     }
+}
 
-    if (valid) {
-        float *dst = a.state + (size_t)i * S + (size_t)sub * E;
+template <int S>
+__device__ __forceinline__ void synth_store(const SynthArgs &a, const f2 (&P)[SynthShape<S>::H], uint32_t len, uint32_t rc,
+                                            uint32_t i, uint32_t sub)
+{
+    constexpr int E = SynthShape<S>::E, H = SynthShape<S>::H;
+    float xo[E];
 #pragma unroll
-        for (int v = 0; v < E / 4; ++v)
-            *reinterpret_cast<float4 *>(dst + 4 * v) = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
-        if (a.next_obs) {
-            float *nd = a.next_obs + (size_t)i * S + (size_t)sub * E;
+    for (int j = 0; j < H; ++j) { xo[j] = lo(P[j]); xo[j + H] = hi(P[j]); }
+    float4 *dst = reinterpret_cast<float4 *>(a.state + (size_t)i * S + (size_t)sub * E);
 #pragma unroll
-            for (int v = 0; v < E / 4; ++v)
-                *reinterpret_cast<float4 *>(nd + 4 * v) = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
-        }
-        if (sub == 0) { a.ep_len[i] = len; a.reset_count[i] = rc; }
+    for (int v = 0; v < E / 4; ++v) dst[v] = make_float4(xo[4 * v], xo[4 * v + 1], xo[4 * v + 2], xo[4 * v + 3]);
+    if (a.next_obs) {
+        float4 *nd = reinterpret_cast<float4 *>(a.next_obs + (size_t)i * S + (size_t)sub * E);
+#pragma unroll
+        for (int v = 0; v < E / 4; ++v) nd[v] = make_float4(xo[4 * v], xo[4 * v + 1], xo[4 * v + 2], xo[4 * v + 3]);
     }
+    if (sub == 0) { a.ep_len[i] = len; a.reset_count[i] = rc; }
+}
+
+// One tile (THREADS chunks) per CTA; each thread loads its chunk straight into registers.  (A persistent
+// variant with a cp.async ring of shared-memory stages was measured for K = 1 and was slower: at K = 1
+// the launch is bound by instruction issue per tile, not by bytes in flight.)
+template <int S>
+__global__ void __launch_bounds__(SynthShape<S>::THREADS)
+rollout_synth_kernel(const __grid_constant__ SynthArgs a)
+{
+    using Sh = SynthShape<S>;
+    constexpr int E = Sh::E, H = Sh::H, L = Sh::L;
+    __shared__ SynthExchange<Sh::WARPS> xc;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t sub = tid % L;
+    uint32_t i = blockIdx.x * (uint32_t)Sh::ENVS_PER_CTA + tid / L;
+    const bool valid = i < a.n;                         // tail threads compute on env n-1 and store nothing
+    if (!valid) i = a.n - 1u;
+
+    f2 P[H];
+    {
+        float xin[E];
+        const float4 *src = reinterpret_cast<const float4 *>(a.state + (size_t)i * S + (size_t)sub * E);
+#pragma unroll
+        for (int v = 0; v < E / 4; ++v) { const float4 f = src[v]; xin[4 * v] = f.x; xin[4 * v + 1] = f.y; xin[4 * v + 2] = f.z; xin[4 * v + 3] = f.w; }
+#pragma unroll
+        for (int j = 0; j < H; ++j) P[j] = pk(xin[j], xin[j + H]);
+    }
+    uint32_t len = a.ep_len[i], rc = a.reset_count[i];
+    synth_steps<S>(a, P, len, rc, i, valid, sub, xc);
+    if (valid) synth_store<S>(a, P, len, rc, i, sub);
 }
 
 template <int S>
 static cudaError_t launch_synth_t(const SynthArgs &a, cudaStream_t st)
 {
     using Sh = SynthShape<S>;
-    const uint32_t blocks = (a.n + Sh::ENVS_PER_CTA - 1u) / Sh::ENVS_PER_CTA;
-    rollout_synth_kernel<S><<<blocks, Sh::THREADS, 0, st>>>(a);
+    const uint32_t ntiles = (a.n + Sh::ENVS_PER_CTA - 1u) / Sh::ENVS_PER_CTA;
+    rollout_synth_kernel<S><<<ntiles, Sh::THREADS, 0, st>>>(a);
     return cudaGetLastError();
 }
 
