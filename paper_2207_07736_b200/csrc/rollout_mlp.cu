@@ -40,6 +40,14 @@ __device__ __forceinline__ void stage_mlp2(const float *__restrict__ p, MlpSmem2
     __syncthreads();
 }
 
+#ifndef MLP_JB
+#define MLP_JB 8
+#endif
+#ifndef MLP_MINBLOCKS
+#define MLP_MINBLOCKS 2
+#endif
+constexpr int kJB = MLP_JB;        // hidden units of layer 2 advanced together (accumulators live in registers)
+
 __device__ __forceinline__ const float4 &ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
 
 // Logits of two observations: la = (logit0, logit1) of obs A, lb of obs B.
@@ -71,23 +79,27 @@ __device__ __forceinline__ void mlp_logits2(const float4 oa, const float4 ob, co
     la = pk(s.b3.x, s.b3.y);
     lb = la;
 #pragma unroll 1
-    for (int jb = 0; jb < 64; jb += 8) {
-        f2 ca[4], cb[4];
-        {
-            const float4 u = ld4(&s.b2[jb]), v = ld4(&s.b2[jb + 4]);
-            ca[0] = pk(u.x, u.y); ca[1] = pk(u.z, u.w); ca[2] = pk(v.x, v.y); ca[3] = pk(v.z, v.w);
-            cb[0] = ca[0]; cb[1] = ca[1]; cb[2] = ca[2]; cb[3] = ca[3];
+    for (int jb = 0; jb < 64; jb += kJB) {
+        f2 ca[kJB / 2], cb[kJB / 2];
+#pragma unroll
+        for (int v = 0; v < kJB / 4; ++v) {
+            const float4 u = ld4(&s.b2[jb + 4 * v]);
+            ca[2 * v] = pk(u.x, u.y); ca[2 * v + 1] = pk(u.z, u.w);
+            cb[2 * v] = ca[2 * v]; cb[2 * v + 1] = ca[2 * v + 1];
         }
 #pragma unroll
         for (int k = 0; k < 64; ++k) {
-            const float4 u = ld4(&s.w2t[k * 64 + jb]), v = ld4(&s.w2t[k * 64 + jb + 4]);
-            const f2 w0 = pk(u.x, u.y), w1 = pk(u.z, u.w), w2 = pk(v.x, v.y), w3 = pk(v.z, v.w);
             const f2 da = splat(ha[k]), db = splat(hb[k]);
-            ca[0] = fma2(w0, da, ca[0]); ca[1] = fma2(w1, da, ca[1]); ca[2] = fma2(w2, da, ca[2]); ca[3] = fma2(w3, da, ca[3]);
-            cb[0] = fma2(w0, db, cb[0]); cb[1] = fma2(w1, db, cb[1]); cb[2] = fma2(w2, db, cb[2]); cb[3] = fma2(w3, db, cb[3]);
+#pragma unroll
+            for (int v = 0; v < kJB / 4; ++v) {
+                const float4 u = ld4(&s.w2t[k * 64 + jb + 4 * v]);
+                const f2 w0 = pk(u.x, u.y), w1 = pk(u.z, u.w);
+                ca[2 * v] = fma2(w0, da, ca[2 * v]); ca[2 * v + 1] = fma2(w1, da, ca[2 * v + 1]);
+                cb[2 * v] = fma2(w0, db, cb[2 * v]); cb[2 * v + 1] = fma2(w1, db, cb[2 * v + 1]);
+            }
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kJB / 2; ++i) {
             const f2 ta = tanh2(ca[i]), tb = tanh2(cb[i]);
             const float2 wl = s.w3[jb + 2 * i], wh = s.w3[jb + 2 * i + 1];
             la = fma2(pk(wl.x, wl.y), splat(lo(ta)), la);
@@ -111,7 +123,7 @@ __device__ __forceinline__ int sample_pair(f2 l, uint32_t w)
 
 constexpr int kMlp2Threads = 128;  // 4 warps x 64 envs
 
-__global__ void __launch_bounds__(kMlp2Threads, 2)
+__global__ void __launch_bounds__(kMlp2Threads, MLP_MINBLOCKS)
 rollout_cartpole_mlp_kernel(const __grid_constant__ S4Args a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];

@@ -197,17 +197,40 @@ __device__ __forceinline__ f2 exp2_core(f2 y)
     return mul2(p, scale);
 }
 
+// exp of two arguments in [0, 88] whose reduced exponent n is >= 0: p * 2^n is formed by adding n to the
+// exponent field of p (p lies in [0.7, 1.42], so the sum stays a normal number and equals the product
+// exactly); this frees one FMA-pipe slot per pair.
+__device__ __forceinline__ f2 exp2_nonneg(f2 y)
+{
+    const f2 magic = splat(kRoundMagic);
+    const f2 t = mul2(y, splat(fbits(0x3FB8AA3Bu)));
+    const f2 nb = add2(t, magic);
+    const f2 nn = sub2(magic, nb);
+    f2 r = fma2(nn, splat(fbits(0x3F317218u)), y);
+    r = fma2(nn, splat(fbits(0xB102E308u)), r);
+    f2 p = fma2(splat(fbits(0x39500D01u)), r, splat(fbits(0x3AB60B61u)));
+    p = fma2(p, r, splat(fbits(0x3C088889u)));
+    p = fma2(p, r, splat(fbits(0x3D2AAAABu)));
+    p = fma2(p, r, splat(fbits(0x3E2AAAABu)));
+    p = fma2(p, r, splat(0.5f));
+    p = fma2(p, r, splat(1.0f));
+    p = fma2(p, r, splat(1.0f));
+    return pk(__uint_as_float(__float_as_uint(lo(p)) + (__float_as_uint(lo(nb)) << 23)),
+              __uint_as_float(__float_as_uint(hi(p)) + (__float_as_uint(hi(nb)) << 23)));
+}
+
 // tanh of two arguments.  d = exp(2|x|) + 1 lies in [2, 2^27) whenever the result is used, where one
 // Newton step from the hardware reciprocal is the correctly rounded reciprocal (checked exhaustively
 // on the device by the library's arithmetic self-check), so 1 - 2/d is one more fused multiply-add.
+// Sign flips and the 2^n scaling run on the integer pipe; the FMA pipe is the one this kernel fills.
 __device__ __forceinline__ f2 tanh2(f2 x)
 {
     const float xa = lo(x), xb = hi(x);
     const float aa = fabsf(xa), ab = fabsf(xb);
-    const f2 a = pk(aa, ab);
-    const f2 e = exp2_core(add2(a, a));
+    const f2 a = pk(aa, ab);                                        // above 9 whatever comes out is replaced below
+    const f2 e = exp2_nonneg(add2(a, a));
     const f2 d = add2(e, splat(1.0f));
-    const f2 nd = fma2(e, splat(-1.0f), splat(-1.0f));            // -d exactly
+    const f2 nd = pk(-lo(d), -hi(d));
     const f2 y0 = pk(rcp_approx(lo(d)), rcp_approx(hi(d)));
     const f2 y1 = fma2(y0, fma2(nd, y0, splat(1.0f)), y0);
     const f2 t = fma2(splat(-2.0f), y1, splat(1.0f));
