@@ -118,13 +118,13 @@ def physical_gpu_index(local_index):
 # ------------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ------------------------------------------------------------------------------------------------
-def oracle_rate(w, budget_s, n_sample=None):
+def oracle_rate(w, budget_s, n_sample=None, compute_factor=1):
     """env-steps/s of the single-threaded oracle on a bounded sample of the workload."""
     import oracle
     n = n_sample or min(w.n_envs, 256 if w.mlp_seed is not None else max(4, 4096 * 4 // w.state_dim))
     params = None if w.mlp_seed is None else inputs.mlp_params(w.mlp_seed)
     ids = inputs.sample_env_ids(3, w.n_envs, n)
-    sim = oracle.OracleSim(w.env_kind, state_dim=w.state_dim, seed=w.seed, env_ids=ids)
+    sim = oracle.OracleSim(w.env_kind, state_dim=w.state_dim, seed=w.seed, env_ids=ids, compute_factor=compute_factor)
     want = ("obs", "act", "rew", "done") if w.trajectory else ()
     steps = 0
     t0 = time.perf_counter()
@@ -145,11 +145,11 @@ def run_reference(args, w):
         return 0
     per_step_budget = max(0.2, min(5.0, 60.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
-        oracle_rate(w, per_step_budget)
+        oracle_rate(w, per_step_budget, compute_factor=args.compute_factor)
     rates, sample = [], ""
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        r, sample = oracle_rate(w, per_step_budget)
+        r, sample = oracle_rate(w, per_step_budget, compute_factor=args.compute_factor)
         rates.append(r)
     wall = time.perf_counter() - t0
     v = statistics.mean(rates)
@@ -197,7 +197,7 @@ def run_gpu(args, w):
 
     env_offset, n = shard.env_range(rank, world, w.n_envs)
     K = args.k_fused or max(w.k_sweep)
-    sim = binding.Sim(w.env_kind, n, w.state_dim, w.seed, device=dev, env_offset=env_offset)
+    sim = binding.Sim(w.env_kind, n, w.state_dim, w.seed, device=dev, env_offset=env_offset, compute_factor=args.compute_factor)
     d_params = None if w.mlp_seed is None else torch.from_numpy(inputs.mlp_params(w.mlp_seed)).to(dev)
     out = sim.alloc_outputs(w.T) if w.trajectory else {}
     traj_bytes = sum(t.numel() * t.element_size() for t in out.values() if t is not None)
@@ -242,6 +242,10 @@ def run_gpu(args, w):
     k_per_launch = min(K, w.T)
     bytes_per_launch = bytes_per_env_step * n * k_per_launch
     fl_nom, fl_exp = nominal_flops_per_env_step(w)
+    if args.compute_factor != 1:                                   # only the dynamics repeat, not the policy
+        dyn = nominal_flops_per_env_step(w if w.mlp_seed is None else inputs.WORKLOADS["cfg2"])
+        fl_nom += (args.compute_factor - 1) * dyn[0]
+        fl_exp += (args.compute_factor - 1) * dyn[1]
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     fp32_peak_tflops = 2 * FP32_LANES_PER_SM * sms * sm_max_mhz * 1e6 / 1e12
     t_hbm = bytes_per_env_step / (hbm_peak * 1e9)
@@ -316,7 +320,7 @@ def run_gpu(args, w):
 
     cpu = None
     if not args.no_cpu and world == 1:
-        v, sample = oracle_rate(w, args.cpu_seconds)
+        v, sample = oracle_rate(w, args.cpu_seconds, compute_factor=args.compute_factor)
         cpu = {"value": v, "unit": "env-steps/s", "cores": 1, "kind": "oracle", "sample": sample,
                "host_cores_available": os.cpu_count()}
 
@@ -325,7 +329,7 @@ def run_gpu(args, w):
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "env": ["cartpole", "acrobot", "synthetic"][w.env_kind], "n_envs_per_gpu": n, "T": w.T,
-                   "state_dim": w.state_dim, "k_fused": K, "policy": "mlp_4_64_64_2" if w.mlp_seed is not None else "uniform_random",
+                   "state_dim": w.state_dim, "k_fused": K, "compute_factor": args.compute_factor, "policy": "mlp_4_64_64_2" if w.mlp_seed is not None else "uniform_random",
                    "trajectory_bytes_per_step": traj_bytes,
                    "l2": "each step writes %.2f GB of trajectory (> 126 MB L2); no flush between steps" % (traj_bytes / 1e9) if traj_bytes > 2e8
                    else "state (%.2f GB) streamed from HBM every launch" % (n * w.state_dim * 4 / 1e9),
@@ -334,6 +338,32 @@ def run_gpu(args, w):
         "k_sweep": sweep,
     }
     print(json.dumps(line), flush=True)
+    return 0
+
+
+def run_grid(args):
+    """Fusion speedup over the simulator-complexity grid of the paper (Section 4.2): state factor S and
+    compute factor C of the synthetic simulator, K fused steps, normalised to K = 1.  One JSON line per (S, C)."""
+    import dataclasses
+    import torch
+    from paper_2207_07736_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --grid needs a CUDA device")
+    T, ks = 64, (1, 8, 64)
+    for S in (4, 64, 512, 4096):
+        n = (128 << 20) // S                                   # 512 MiB of state: streams from HBM at K = 1
+        for C in (1, 4, 16, 64):
+            sim = binding.Sim(inputs.SYNTH, n, S, 0, compute_factor=C)
+            w = dataclasses.replace(inputs.WORKLOADS["cfg5_S%d" % S], n_envs=n, T=T)
+            row = {"grid": "simulator_complexity", "S": S, "C": C, "n_envs": n, "T": T, "k": {}}
+            for k in ks:
+                time_rollouts(torch, sim, w, k, 1, None, {})
+                ms = statistics.median(time_rollouts(torch, sim, w, k, 3, None, {}))
+                row["k"][str(k)] = {"ms": ms, "env_steps_per_sec": n * T / (ms * 1e-3)}
+            for k in ks:
+                row["k"][str(k)]["fusion_speedup_vs_k1"] = row["k"]["1"]["ms"] / row["k"][str(k)]["ms"]
+            print(json.dumps(row), flush=True)
+            sim.close()
     return 0
 
 
@@ -351,6 +381,8 @@ def main():
     ap.add_argument("--traffic-bytes", type=float, default=None, help="ncu dram bytes per launch, if captured for this shape")
     ap.add_argument("--n-envs", type=int, default=0, help="override the workload's env count (profiling on a reduced case)")
     ap.add_argument("--T", type=int, default=0, help="override the workload's step count (profiling on a reduced case)")
+    ap.add_argument("--compute-factor", type=int, default=1, help="dynamics iterations per recorded step (the paper's knob C)")
+    ap.add_argument("--grid", action="store_true", help="fusion speedup over the S x C x K simulator-complexity grid (synthetic simulator)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -361,6 +393,8 @@ def main():
     if args.n_envs or args.T:
         import dataclasses
         w = dataclasses.replace(w, name=w.name + "_reduced", n_envs=args.n_envs or w.n_envs, T=args.T or w.T)
+    if args.grid:
+        return run_grid(args)
     if args.impl == "reference":
         return run_reference(args, w)
     return run_gpu(args, w)

@@ -70,6 +70,14 @@ int sim_set_stream(sim_t *s, void *cuda_stream);
  * offset + n_envs must not exceed 2^32.  Takes effect at the next sim_reset. */
 int sim_set_env_offset(sim_t *s, uint64_t env_offset);
 
+/* sim_set_compute_factor -- the paper's compute-factor knob C (Section 4.2, "increases the compute
+ * requirements ... by increasing the number of simulation iterations"): one recorded step becomes C
+ * iterations of the env's dynamics update under the step's one action (for Acrobot each iteration is a
+ * full RK4 step with wrap and clip); reward, the done test and ep_len refer to the state after the last
+ * iteration, and the trajectory still has one row per recorded step.  1 <= C <= 65536, default 1 (the
+ * plain simulator).  Applies to every later sim_step / sim_rollout of the handle. */
+int sim_set_compute_factor(sim_t *s, int compute_factor);
+
 /* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env. */
 int sim_reset(sim_t *s);
 

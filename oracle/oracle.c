@@ -394,7 +394,7 @@ ORACLE_API int oracle_sample_action(const float logits[2], uint32_t w)
  * next_obs, if not NULL, is [T,n_sel,S]: the state after step t and after auto-reset.
  * Returns 0, or -1 on bad arguments.
  * ---------------------------------------------------------------------------------- */
-ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
+ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_factor,
                               int64_t n_sel, const uint32_t *env_ids,
                               float *state, uint32_t *ep_len, uint32_t *reset_count,
                               uint64_t t0, int T,
@@ -405,6 +405,7 @@ ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
     if (env_kind < 0 || env_kind > 2 || S < 4 || S > 4096 || (S & (S - 1)) || T < 0 || n_sel < 0) return -1;
     if (env_kind != ENV_SYNTH && S != 4) return -1;
     if (policy_params && env_kind != ENV_CARTPOLE) return -1;
+    if (compute_factor < 1) return -1;
     float cur[4096], nxt[4096], scratch[4096];
     for (int64_t e = 0; e < n_sel; ++e) {
         uint32_t env = env_ids[e];
@@ -427,24 +428,25 @@ ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
                 act = oracle_random_action(env_kind, w);
             }
 
-            int done; float rew;
-            if (env_kind == ENV_CARTPOLE) {
-                act = act ? 1 : 0;
-                done = oracle_cartpole_step(cur, act, nxt);
-                rew = 1.0f;
-                len += 1;
-            } else if (env_kind == ENV_ACROBOT) {
-                if (act < 0) act = 0;
-                if (act > 2) act = 2;
-                int goal = oracle_acrobot_step(cur, act, nxt);
-                len += 1;
+            /* compute factor C (paper Section 4.2): the dynamics update is iterated C times with the
+             * action held; reward, done and ep_len refer to the state after the last iteration */
+            int done = 0; float rew;
+            if (env_kind == ENV_CARTPOLE) act = act ? 1 : 0;
+            else if (env_kind == ENV_ACROBOT) act = act < 0 ? 0 : (act > 2 ? 2 : act);
+            else act = act ? 1 : 0;
+            for (int c = 0; c < compute_factor; ++c) {
+                if (c > 0) memcpy(cur, nxt, sizeof(float) * (size_t)S);
+                if (env_kind == ENV_CARTPOLE) done = oracle_cartpole_step(cur, act, nxt);
+                else if (env_kind == ENV_ACROBOT) done = oracle_acrobot_step(cur, act, nxt);
+                else done = oracle_synth_step(cur, S, act, nxt, scratch);
+            }
+            len += 1;
+            if (env_kind == ENV_ACROBOT) {
+                int goal = done;
                 done = goal | (len >= 500u);
                 rew = goal ? 0.0f : -1.0f;
             } else {
-                act = act ? 1 : 0;
-                done = oracle_synth_step(cur, S, act, nxt, scratch);
                 rew = 1.0f;
-                len += 1;
             }
             if (out_act) out_act[row] = (int8_t)act;
             if (out_rew) out_rew[row] = rew;
@@ -463,6 +465,19 @@ ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
         ep_len[e] = len; reset_count[e] = rc;
     }
     return 0;
+}
+
+/* The plain simulator: compute factor 1. */
+ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
+                              int64_t n_sel, const uint32_t *env_ids,
+                              float *state, uint32_t *ep_len, uint32_t *reset_count,
+                              uint64_t t0, int T,
+                              const float *policy_params, const int8_t *given_actions,
+                              float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done,
+                              float *next_obs)
+{
+    return oracle_rollout_c(env_kind, S, seed, 1, n_sel, env_ids, state, ep_len, reset_count, t0, T,
+                            policy_params, given_actions, out_obs, out_act, out_rew, out_done, next_obs);
 }
 
 /* Initial condition (draw #0, zeroed counters) for a list of env indices. */

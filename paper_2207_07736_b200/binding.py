@@ -23,6 +23,7 @@ SIGNATURES = {
     "sim_destroy": (C.c_int, [C.c_void_p]),
     "sim_set_stream": (C.c_int, [C.c_void_p, C.c_void_p]),
     "sim_set_env_offset": (C.c_int, [C.c_void_p, C.c_uint64]),
+    "sim_set_compute_factor": (C.c_int, [C.c_void_p, C.c_int]),
     "sim_reset": (C.c_int, [C.c_void_p]),
     "sim_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "sim_rollout": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -101,6 +102,10 @@ def sim_set_env_offset(h, env_offset):
     _check(lib().sim_set_env_offset(h, env_offset), h)
 
 
+def sim_set_compute_factor(h, compute_factor):
+    _check(lib().sim_set_compute_factor(h, compute_factor), h)
+
+
 def sim_reset(h):
     _check(lib().sim_reset(h), h)
 
@@ -159,7 +164,7 @@ def sim_launch_count(h):
 class Sim:
     """Owning wrapper of one handle, with torch tensors for the outputs (memory plumbing only)."""
 
-    def __init__(self, env_kind, n_envs, state_dim=4, seed=0, device="cuda:0", env_offset=0):
+    def __init__(self, env_kind, n_envs, state_dim=4, seed=0, device="cuda:0", env_offset=0, compute_factor=1):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -169,6 +174,8 @@ class Sim:
             if env_offset:
                 sim_set_env_offset(self.h, env_offset)
                 sim_reset(self.h)
+            if compute_factor != 1:
+                sim_set_compute_factor(self.h, compute_factor)
         self.use_stream(None)
 
     def use_stream(self, stream):

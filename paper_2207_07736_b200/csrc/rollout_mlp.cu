@@ -162,8 +162,9 @@ rollout_cartpole_mlp_kernel(const __grid_constant__ S4Args a)
             f2 la, lb;
             mlp_logits2(A, B, ms, la, lb);
             const int act_a = sample_pair(la, wa), act_b = sample_pair(lb, wb);
-            const bool da = cartpole_step(A, act_a != 0);
-            const bool db = cartpole_step(B, act_b != 0);
+            bool da = cartpole_step(A, act_a != 0);
+            bool db = cartpole_step(B, act_b != 0);
+            for (int c = 1; c < a.C; ++c) { da = cartpole_step(A, act_a != 0); db = cartpole_step(B, act_b != 0); }   // compute factor
             len_a += 1u; len_b += 1u;
             if (sa_act) __stcs(a.out_act + row, (int8_t)act_a);
             if (sb_act) __stcs(a.out_act + row + 32, (int8_t)act_b);

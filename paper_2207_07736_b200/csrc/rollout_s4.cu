@@ -17,18 +17,22 @@ __device__ __forceinline__ int random_action(uint32_t w)
     return ENV == ENV_ACROBOT ? (int)__umulhi(w, 3u) : (int)(w >> 31);
 }
 
+// One recorded step: C iterations of the dynamics under one action (C = 1: the plain simulator);
+// reward, done and ep_len refer to the state after the last iteration.
 template <int ENV>
-__device__ __forceinline__ bool env_step(float4 &s, int &act, uint32_t &len, float &rew)
+__device__ __forceinline__ bool env_step(float4 &s, int &act, uint32_t &len, float &rew, int C)
 {
     if (ENV == ENV_CARTPOLE) {
         act = act ? 1 : 0;
-        const bool done = cartpole_step(s, act != 0);
+        bool done = cartpole_step(s, act != 0);
+        for (int c = 1; c < C; ++c) done = cartpole_step(s, act != 0);
         len += 1u;
         rew = 1.0f;
         return done;
     } else {
         act = min(max(act, 0), 2);
-        const bool goal = acrobot_step(s, act);
+        bool goal = acrobot_step(s, act);
+        for (int c = 1; c < C; ++c) goal = acrobot_step(s, act);
         len += 1u;
         rew = goal ? 0.0f : -1.0f;
         return goal | (len >= 500u);
@@ -70,7 +74,7 @@ rollout_s4_kernel(const __grid_constant__ S4Args a)
             }
 
             float rew;
-            const bool done = env_step<ENV>(s, act, len, rew);
+            const bool done = env_step<ENV>(s, act, len, rew, a.C);
 
             if (a.out_act) __stcs(&a.out_act[row], (int8_t)act);
             if (a.out_rew) __stcs(&a.out_rew[row], rew);

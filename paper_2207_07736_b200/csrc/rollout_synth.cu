@@ -53,7 +53,7 @@ __device__ __forceinline__ f2 sin2(f2 x)
 }
 
 // Shared memory used for the cross-warp exchange of one env (L > 32).
-template <int W> struct SynthExchange { float halo[W]; float sum[W]; };
+template <int W> struct SynthExchange { float halo[2][W]; float sum[W]; };   // halo is double-buffered across iterations
 
 // K steps of one chunk held in registers.  P[j] = (x_j, x_{j+H}).  All threads of a CTA call this
 // together (it contains CTA barriers when an env spans several warps).
@@ -92,36 +92,37 @@ __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[SynthSha
             const int act = a.actions ? (a.actions[i] != 0) : (int)(w >> 31);
             const f2 c = splat(__fmul_rn(fbits(0x3A83126Fu), act ? 1.0f : -1.0f));
 
-            // halo: first element of the next chunk of the same env (wrapping around)
-            const float x0 = lo(P[0]);
-            float halo;
-            if (L == 1) {
-                halo = x0;
-            } else {
-                halo = __shfl_sync(0xFFFFFFFFu, x0, (lane & ~(uint32_t)(LS - 1)) | ((lane + 1u) & (uint32_t)(LS - 1)));
-                if (W > 1) {
-                    if (lane == 0) xc.halo[warp] = x0;
-                    __syncthreads();
-                    if (lane == 31) halo = xc.halo[(warp + 1u) % W];
-                }
-            }
-
-            // Jacobi update: every right-hand side reads pre-step values.  The right neighbours of
-            // pair j = (x_j, x_{j+H}) are pair j+1; the last pair's are (x_H, halo).
-            const f2 wrap = pk(hi(P[0]), halo);
-            const f2 c01 = splat(fbits(0x3C23D70Au));
+            // compute factor: C Jacobi iterations under one action; squares and the done test use the last one
             f2 Q[H];
+            for (int cit = 0; cit < a.C; ++cit) {
+                // halo: first element of the next chunk of the same env (wrapping around)
+                const float x0 = lo(P[0]);
+                float halo;
+                if (L == 1) {
+                    halo = x0;
+                } else {
+                    halo = __shfl_sync(0xFFFFFFFFu, x0, (lane & ~(uint32_t)(LS - 1)) | ((lane + 1u) & (uint32_t)(LS - 1)));
+                    if (W > 1) {
+                        if (lane == 0) xc.halo[cit & 1][warp] = x0;
+                        __syncthreads();
+                        if (lane == 31) halo = xc.halo[cit & 1][(warp + 1u) % W];
+                    }
+                }
+                // Jacobi update: every right-hand side reads pre-iteration values.  The right neighbours of
+                // pair j = (x_j, x_{j+H}) are pair j+1; the last pair's are (x_H, halo).
+                const f2 wrap = pk(hi(P[0]), halo);
+                const f2 c01 = splat(fbits(0x3C23D70Au));
 #pragma unroll
-            for (int j = 0; j < H; ++j) {
-                const f2 right = j + 1 < H ? P[j + 1] : wrap;
-                const f2 z = sin2(add2(P[j], right));
-                Q[j] = add2(fma2(c01, z, P[j]), c);
+                for (int j = 0; j < H; ++j) {
+                    const f2 right = j + 1 < H ? P[j + 1] : wrap;
+                    const f2 z = sin2(add2(P[j], right));
+                    Q[j] = add2(fma2(c01, z, P[j]), c);
+                }
+#pragma unroll
+                for (int j = 0; j < H; ++j) P[j] = Q[j];
             }
 #pragma unroll
-            for (int j = 0; j < H; ++j) {
-                P[j] = Q[j];
-                Q[j] = mul2(Q[j], Q[j]);
-            }
+            for (int j = 0; j < H; ++j) Q[j] = mul2(P[j], P[j]);
 #pragma unroll
             for (int wdt = 1; wdt < H; wdt <<= 1)
 #pragma unroll

@@ -18,6 +18,7 @@ struct sim {
     uint64_t seed;
     uint64_t env_offset;
     uint64_t t;
+    int compute_factor;
     int device;
     cudaStream_t stream;
     float *state;
@@ -102,6 +103,7 @@ SIM_API int sim_create(sim_t **out, int env_kind, int64_t n_envs, int state_dim,
     if (!s) return SIM_ENOMEM;
     memset(s, 0, sizeof(*s));
     s->env_kind = env_kind; s->S = state_dim; s->n = (uint32_t)n_envs; s->seed = seed;
+    s->compute_factor = 1;
     expand_keys(seed, s->rk);
     cudaError_t e = cudaGetDevice(&s->device);
     if (e == cudaSuccess) e = cudaMalloc(&s->state, (size_t)n_envs * (size_t)state_dim * sizeof(float));
@@ -142,6 +144,13 @@ SIM_API int sim_set_env_offset(sim_t *s, uint64_t env_offset)
     return SIM_OK;
 }
 
+SIM_API int sim_set_compute_factor(sim_t *s, int compute_factor)
+{
+    if (!s || compute_factor < 1 || compute_factor > 65536) return SIM_EINVAL;
+    s->compute_factor = compute_factor;
+    return SIM_OK;
+}
+
 SIM_API int sim_reset(sim_t *s)
 {
     if (!s) return SIM_EINVAL;
@@ -160,17 +169,17 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
     if (s->env_kind == SIM_SYNTH) {
         SynthArgs a;
         a.state = s->state; a.ep_len = s->ep_len; a.reset_count = s->reset_count;
-        a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K;
+        a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = s->compute_factor;
         a.out_obs = obs; a.out_act = act; a.out_rew = rew; a.out_done = done;
         a.actions = d_actions; a.next_obs = next_obs; a.rk = s->rk;
         CU(s, launch_synth(s->S, a, s->stream));
     } else {
         S4Args a;
         a.state = reinterpret_cast<float4 *>(s->state); a.ep_len = s->ep_len; a.reset_count = s->reset_count;
-        a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K;
+        a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = s->compute_factor;
         a.out_obs = reinterpret_cast<float4 *>(obs); a.out_act = act; a.out_rew = rew; a.out_done = done;
         a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.rk = s->rk;
-        if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM)
+        if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM && s->compute_factor == 1)
             CU(s, launch_cartpole_random(a, s->stream));
         else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP)
             CU(s, launch_cartpole_mlp(a, s->stream));

@@ -19,6 +19,7 @@ struct S4Args {
     uint32_t tb0;             // (t0 >> 2) truncated to 32 bits: Philox counter word of the first action block
     int phase;                // t0 & 3
     int K;                    // steps in this launch
+    int C;                    // compute factor: dynamics iterations per recorded step (>= 1)
     float4 *out_obs;          // [K, n] or nullptr
     int8_t *out_act;          // [K, n] or nullptr
     float *out_rew;           // [K, n] or nullptr
@@ -39,6 +40,7 @@ struct SynthArgs {
     uint32_t tb0;
     int phase;
     int K;
+    int C;                    // compute factor
     float *out_obs;           // [K, n, S] or nullptr
     int8_t *out_act;
     float *out_rew;

@@ -94,7 +94,7 @@ int sim_rollout_noalloc(int env_kind, int64_t n_envs, int state_dim, uint64_t se
         if (env_kind == SIM_SYNTH) {
             SynthArgs a;
             a.state = state; a.ep_len = ep_len; a.reset_count = reset_count; a.n = (uint32_t)n; a.env_offset = 0u;
-            a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k;
+            a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k; a.C = 1;
             a.out_obs = out_obs ? out_obs + r0 * S : nullptr; a.out_act = out_act ? out_act + r0 : nullptr;
             a.out_rew = out_rew ? out_rew + r0 : nullptr; a.out_done = out_done ? out_done + r0 : nullptr;
             a.actions = nullptr; a.next_obs = nullptr; a.rk = rk;
@@ -102,7 +102,7 @@ int sim_rollout_noalloc(int env_kind, int64_t n_envs, int state_dim, uint64_t se
         } else {
             S4Args a;
             a.state = reinterpret_cast<float4 *>(state); a.ep_len = ep_len; a.reset_count = reset_count; a.n = (uint32_t)n; a.env_offset = 0u;
-            a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k;
+            a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k; a.C = 1;
             a.out_obs = out_obs ? reinterpret_cast<float4 *>(out_obs) + r0 : nullptr; a.out_act = out_act ? out_act + r0 : nullptr;
             a.out_rew = out_rew ? out_rew + r0 : nullptr; a.out_done = out_done ? out_done + r0 : nullptr;
             a.actions = nullptr; a.next_obs = nullptr; a.params = d_policy_params; a.rk = rk;

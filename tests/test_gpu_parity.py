@@ -153,6 +153,56 @@ def test_checkpoint_resume_and_split_rollout():
     assert torch.equal(a.state(), c.state())
 
 
+@pytest.mark.parametrize("kind,S", [(oracle.CARTPOLE, 4), (oracle.ACROBOT, 4), (oracle.SYNTH, 64)])
+def test_large_step_index_and_counter_restore(kind, S):
+    """The action counter uses (t >> 2) truncated to 32 bits; a handle restored at a huge t, at every
+    phase of the 4-step block, must keep matching the oracle."""
+    torch = torch_cuda()
+    for t0 in ((1 << 34) + 1, (1 << 32) - 3, 7):
+        sim = binding.Sim(kind, 130, S, 13)
+        orc = oracle.OracleSim(kind, 130, S, 13)
+        ep, rc, _ = sim.counters()
+        sim.set_counters(ep, rc, t0)
+        orc.t = t0
+        out = sim.rollout(21, 5)
+        torch.cuda.synchronize()
+        ref = orc.rollout(21)
+        compare_rollout(out, sim, ref, orc, what="t0=%d" % t0)
+
+
+@pytest.mark.parametrize("C", [2, 5])
+def test_compute_factor_all_envs(C):
+    """The paper's compute-factor knob: C dynamics iterations per recorded step, on every kernel."""
+    torch = torch_cuda()
+    cases = [(oracle.CARTPOLE, 4, 300, 90, 30, None), (oracle.CARTPOLE, 4, 200, 40, 8, inputs.mlp_params(1, 0.2)),
+             (oracle.ACROBOT, 4, 257, 120, 50, None), (oracle.SYNTH, 4, 500, 20, 7, None), (oracle.SYNTH, 64, 77, 20, 20, None),
+             (oracle.SYNTH, 512, 40, 12, 5, None), (oracle.SYNTH, 4096, 6, 9, 4, None)]
+    for kind, S, n, T, K, params in cases:
+        sim = binding.Sim(kind, n, S, 17, compute_factor=C)
+        orc = oracle.OracleSim(kind, n, S, 17, compute_factor=C)
+        if kind == oracle.SYNTH:
+            st = orc.state.copy()
+            st[::4] = 2.0                                   # some envs cross the threshold within a few iterations
+            orc.state[:] = st
+            sim.set_state(torch.from_numpy(st).cuda())
+        d_params = None if params is None else torch.from_numpy(params).cuda()
+        out = sim.rollout(T, K, d_params)
+        torch.cuda.synchronize()
+        ref = orc.rollout(T, policy_params=params)
+        compare_rollout(out, sim, ref, orc, what="C=%d kind=%d S=%d" % (C, kind, S))
+        # given-action steps use the same factor
+        acts = inputs.forced_actions(2, 3, n, 3 if kind == oracle.ACROBOT else 2)
+        for t in range(3):
+            nxt, rew, done = sim.step(torch.from_numpy(acts[t]).cuda())
+            o_nxt, o_rew, o_done = orc.step(acts[t])
+            assert_same_bits(to_np(nxt), o_nxt, "C step next_obs")
+            assert_same_bits(to_np(done), o_done, "C step done")
+    L = binding.lib()
+    sim = binding.Sim(oracle.CARTPOLE, 8)
+    assert L.sim_set_compute_factor(sim.h, 0) == binding.SIM_EINVAL and L.sim_set_compute_factor(sim.h, 65537) == binding.SIM_EINVAL
+    assert L.sim_set_compute_factor(None, 2) == binding.SIM_EINVAL
+
+
 def test_null_outputs_and_reset():
     torch = torch_cuda()
     sim = binding.Sim(oracle.CARTPOLE, 777, 4, 1)

@@ -82,3 +82,30 @@ def test_workload_table_shapes():
         c = w["cfg5_S%d" % S]
         assert c.n_envs * S * 4 == 4 << 30 and not c.trajectory
     assert inputs.mlp_params(1).shape == (4610,) and np.all(inputs.mlp_params(1)[256:320] == 0)
+
+
+def test_compute_factor_is_iterated_dynamics_with_the_action_held():
+    """Compute factor C (the paper's simulator-complexity knob): one recorded step = C dynamics
+    iterations under one action.  Where no episode ends, that equals C plain steps with the action repeated."""
+    for kind, S, T, C in [(oracle.CARTPOLE, 4, 3, 2), (oracle.ACROBOT, 4, 30, 3), (oracle.SYNTH, 16, 12, 4)]:
+        n = 24
+        fat = oracle.OracleSim(kind, n, S, seed=8, compute_factor=C)
+        rf = fat.rollout(T)
+        assert not rf["done"].any()
+        plain = oracle.OracleSim(kind, n, S, seed=8)
+        rp = plain.rollout(T * C, actions=np.repeat(rf["act"], C, axis=0))
+        assert not rp["done"].any()
+        assert np.array_equal(rf["obs"], rp["obs"][::C])
+        assert np.array_equal(fat.state, plain.state)
+        assert np.all(fat.ep_len == T) and np.all(plain.ep_len == T * C)      # ep_len counts recorded steps
+        assert fat.t == T
+    # C = 1 is the plain simulator
+    a = oracle.OracleSim(oracle.CARTPOLE, 16, seed=3, compute_factor=1).rollout(60)
+    b = oracle.OracleSim(oracle.CARTPOLE, 16, seed=3).rollout(60)
+    assert all(np.array_equal(a[k], b[k]) for k in ("obs", "act", "rew", "done"))
+    # the done test looks at the state after the last iteration; episodes get shorter in recorded steps
+    fat = oracle.OracleSim(oracle.CARTPOLE, 256, seed=1, compute_factor=4)
+    out = fat.rollout(100)
+    first = np.array([np.flatnonzero(out["done"][:, e])[0] for e in range(256)])
+    assert 1 <= first.min() and first.mean() < 8
+    assert np.array_equal(fat.reset_count, out["done"].sum(0).astype(np.uint32))
