@@ -128,6 +128,8 @@ rollout_cartpole_mlp_kernel(const __grid_constant__ S4Args a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     MlpSmem2 &ms = *reinterpret_cast<MlpSmem2 *>(smem_raw);
+    pdl_wait();                                          // parameters and state may come from the previous launch
+    pdl_release();
     stage_mlp2(a.params, ms);
 
     const uint32_t lane = threadIdx.x & 31u;
@@ -200,8 +202,7 @@ cudaError_t launch_cartpole_mlp(const S4Args &a, cudaStream_t st)
 {
     const unsigned envs_per_cta = kMlp2Threads * 2;
     const unsigned blocks = (a.n + envs_per_cta - 1u) / envs_per_cta;
-    rollout_cartpole_mlp_kernel<<<blocks, kMlp2Threads, sizeof(MlpSmem2), st>>>(a);
-    return cudaGetLastError();
+    return launch_overlapped(a.K <= kOverlapMaxK, rollout_cartpole_mlp_kernel, dim3(blocks), dim3(kMlp2Threads), sizeof(MlpSmem2), st, a);
 }
 
 cudaError_t launch_policy_logits(const float *obs, int64_t M, const float *params, float *logits, cudaStream_t st)

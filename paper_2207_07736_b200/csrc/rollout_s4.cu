@@ -48,6 +48,8 @@ rollout_s4_kernel(const __grid_constant__ S4Args a)
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= a.n) return;
     const uint32_t env = a.env_offset + i;
+    pdl_wait();
+    pdl_release();
 
     float4 s = a.state[i];
     uint32_t len = a.ep_len[i];
@@ -147,8 +149,7 @@ template <int ENV, int POLICY>
 static cudaError_t launch_s4_t(const S4Args &a, cudaStream_t st)
 {
     const unsigned blocks = (a.n + kS4Threads - 1u) / kS4Threads;
-    rollout_s4_kernel<ENV, POLICY><<<blocks, kS4Threads, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_overlapped(a.K <= kOverlapMaxK, rollout_s4_kernel<ENV, POLICY>, dim3(blocks), dim3(kS4Threads), 0, st, a);
 }
 
 cudaError_t launch_s4(int env_kind, int policy, const S4Args &a, cudaStream_t st)

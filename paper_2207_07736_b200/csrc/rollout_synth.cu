@@ -202,6 +202,8 @@ rollout_synth_kernel(const __grid_constant__ SynthArgs a)
     uint32_t i = blockIdx.x * (uint32_t)Sh::ENVS_PER_CTA + tid / L;
     const bool valid = i < a.n;                         // tail threads compute on env n-1 and store nothing
     if (!valid) i = a.n - 1u;
+    pdl_wait();
+    pdl_release();
 
     f2 P[H];
     {
@@ -222,8 +224,7 @@ static cudaError_t launch_synth_t(const SynthArgs &a, cudaStream_t st)
 {
     using Sh = SynthShape<S>;
     const uint32_t ntiles = (a.n + Sh::ENVS_PER_CTA - 1u) / Sh::ENVS_PER_CTA;
-    rollout_synth_kernel<S><<<ntiles, Sh::THREADS, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_overlapped(a.K <= kOverlapMaxK, rollout_synth_kernel<S>, dim3(ntiles), dim3(Sh::THREADS), 0, st, a);
 }
 
 cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st)

@@ -50,6 +50,31 @@ struct SynthArgs {
     RoundKeys rk;
 };
 
+// Programmatic dependent launch: consecutive rollout launches of one stream overlap their launch
+// latency.  A kernel calls pdl_wait() before its first global-memory access (it returns once every
+// earlier grid of the stream has completed and its writes are visible; a no-op when the launch did not
+// ask for overlap) and pdl_release() right after, which lets the next launch start its own prologue.
+// Overlap is requested for short launches only (K <= kOverlapMaxK): there the launch latency is the
+// cost; for long launches, CTAs of the next grid placed while the current one still fills the SMs end up
+// unevenly spread and the next grid runs slower (measured: +40 % at K = 1000).
+constexpr int kOverlapMaxK = 4;
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_overlapped(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Launchers (each returns the launch error, enqueues on `st`, never synchronises).
 cudaError_t launch_reset(int env_kind, int S, float *state, uint32_t *ep_len, uint32_t *reset_count,
                          uint32_t n, uint32_t env_offset, const RoundKeys &rk, cudaStream_t st);
