@@ -132,13 +132,16 @@ int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t *d_reset
  *   any live handle (it provides the stream). */
 int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits);
 
-/* sim_selfcheck_division -- numerical self-check of the fused CartPole kernel's division (the paper
- * has no counterpart; it exists so a test can prove the kernel's arithmetic on the device it runs
- * on).  For EVERY binary32 denominator the CartPole dynamics can produce (all values in
- * [0.62, 0.67]) it compares the kernel's refined reciprocal with the correctly rounded one, and the
- * kernel's quotient with the IEEE quotient for nums_per_den pseudo-random numerators inside the
- * guarded exponent range.  *h_mismatches (host) = reciprocal mismatches * 2^32 + quotient
- * mismatches; 0 means the kernel's division is the IEEE division on this device.  Synchronises. */
+/* sim_selfcheck_division -- numerical self-check of the divisions inside the fused kernels (the paper
+ * has no counterpart; it exists so a test can prove the kernels' arithmetic on the device they run
+ * on).  The fused CartPole and Acrobot kernels divide by well-conditioned denominators with a refined
+ * hardware reciprocal instead of the general division sequence, and the MLP's tanh uses the refined
+ * reciprocal of exp(2|x|)+1.  For EVERY binary32 value of each denominator range (CartPole [0.62, 0.67];
+ * Acrobot [2.4, 4.6] and [0.5, 1.1]; tanh [2, 2^27]) the refined reciprocal is compared with the correctly
+ * rounded one, and for the division ranges the kernels' quotient is compared with the IEEE quotient for
+ * nums_per_den (CartPole) or nums_per_den/16 (Acrobot) pseudo-random numerators per denominator inside the
+ * guarded exponent range.  *h_mismatches (host) = reciprocal mismatches * 2^32 + quotient mismatches; 0
+ * means the kernels' divisions are the IEEE divisions on this device.  Synchronises. */
 int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_mismatches);
 
 /*

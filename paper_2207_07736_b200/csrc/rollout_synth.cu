@@ -24,34 +24,6 @@ template <int S> struct SynthShape {
     static constexpr int ENVS_PER_CTA = THREADS / L;                    // envs per tile
 };
 
-// sin of two arguments (general quadrant): both polynomials packed, then one select and one sign
-// flip per element.
-__device__ __forceinline__ f2 sin2(f2 x)
-{
-    const f2 magic = splat(kRoundMagic);
-    const f2 t = mul2(x, splat(fbits(0x3F22F983u)));
-    const f2 nb = add2(t, magic);
-    const f2 nk = sub2(magic, nb);
-    f2 r = fma2(nk, splat(fbits(0x3FC90FDBu)), x);
-    r = fma2(nk, splat(fbits(0xB33BBD2Eu)), r);
-    r = fma2(nk, splat(fbits(0xA6F72CEDu)), r);
-    const f2 r2 = mul2(r, r);
-    f2 p = fma2(splat(fbits(0x3638EF1Du)), r2, splat(fbits(0xB9500D01u)));
-    p = fma2(p, r2, splat(fbits(0x3C088889u)));
-    p = fma2(p, r2, splat(fbits(0xBE2AAAABu)));
-    const f2 Sv = fma2(p, mul2(r2, r), r);
-    f2 c = fma2(splat(fbits(0xB493F27Eu)), r2, splat(fbits(0x37D00D01u)));
-    c = fma2(c, r2, splat(fbits(0xBAB60B61u)));
-    c = fma2(c, r2, splat(fbits(0x3D2AAAABu)));
-    c = fma2(c, r2, splat(-0.5f));
-    const f2 Cv = fma2(c, r2, splat(1.0f));
-    const uint32_t qa = __float_as_uint(lo(nb)), qb = __float_as_uint(hi(nb));
-    const float sa = (qa & 1u) ? lo(Cv) : lo(Sv);
-    const float sb = (qb & 1u) ? hi(Cv) : hi(Sv);
-    return pk(__uint_as_float(__float_as_uint(sa) ^ ((qa << 30) & 0x80000000u)),
-              __uint_as_float(__float_as_uint(sb) ^ ((qb << 30) & 0x80000000u)));
-}
-
 // Shared memory used for the cross-warp exchange of one env (L > 32).
 template <int W> struct SynthExchange { float halo[2][W]; float sum[W]; };   // halo is double-buffered across iterations
 

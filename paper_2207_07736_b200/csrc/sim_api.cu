@@ -181,6 +181,8 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
         a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.rk = s->rk;
         if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM && s->compute_factor == 1)
             CU(s, launch_cartpole_random(a, s->stream));
+        else if (s->env_kind == SIM_ACROBOT && policy == POLICY_RANDOM && K > 4)      // short launches: the scalar kernel has the shorter step latency
+            CU(s, launch_acrobot_random(a, s->stream));
         else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP)
             CU(s, launch_cartpole_mlp(a, s->stream));
         else

@@ -80,6 +80,7 @@ cudaError_t launch_reset(int env_kind, int S, float *state, uint32_t *ep_len, ui
                          uint32_t n, uint32_t env_offset, const RoundKeys &rk, cudaStream_t st);
 cudaError_t launch_s4(int env_kind, int policy, const S4Args &a, cudaStream_t st);
 cudaError_t launch_cartpole_random(const S4Args &a, cudaStream_t st);   // CartPole, uniform random policy, packed two-env kernel
+cudaError_t launch_acrobot_random(const S4Args &a, cudaStream_t st);    // Acrobot, uniform random torque, packed two-env kernel
 cudaError_t launch_cartpole_mlp(const S4Args &a, cudaStream_t st);      // CartPole, MLP policy, packed two-env kernel
 cudaError_t launch_division_selfcheck(int nums_per_den, unsigned long long *d_bad, cudaStream_t st);
 cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st);

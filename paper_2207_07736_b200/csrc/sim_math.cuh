@@ -128,6 +128,7 @@ __device__ __forceinline__ f2 add2(f2 a, f2 b) { f2 r; asm("add.rn.f32x2 %0, %1,
 __device__ __forceinline__ f2 sub2(f2 a, f2 b) { f2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
 __device__ __forceinline__ f2 mul2(f2 a, f2 b) { f2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
 
+
 // Quadrant fix-up of one (S, C) polynomial pair: q = k mod 4 in the low bits.
 __device__ __forceinline__ void quadrant_fix(uint32_t q, float S, float C, float &sn, float &cs)
 {
@@ -174,7 +175,96 @@ __device__ __forceinline__ void sincos2(f2 x, f2 &sn, f2 &cs, uint32_t converged
     }
 }
 
+// Polynomial halves of sin/cos for two arguments at once (general quadrant): returns the two
+// polynomial values and the quadrant words; the callers below pick what they need.
+__device__ __forceinline__ void sincos_poly2(f2 x, f2 &S, f2 &C, uint32_t &qa, uint32_t &qb)
+{
+    const f2 magic = splat(kRoundMagic);
+    const f2 t = mul2(x, splat(fbits(0x3F22F983u)));
+    const f2 nb = add2(t, magic);
+    const f2 nk = sub2(magic, nb);
+    f2 r = fma2(nk, splat(fbits(0x3FC90FDBu)), x);
+    r = fma2(nk, splat(fbits(0xB33BBD2Eu)), r);
+    r = fma2(nk, splat(fbits(0xA6F72CEDu)), r);
+    const f2 r2 = mul2(r, r);
+    f2 p = fma2(splat(fbits(0x3638EF1Du)), r2, splat(fbits(0xB9500D01u)));
+    p = fma2(p, r2, splat(fbits(0x3C088889u)));
+    p = fma2(p, r2, splat(fbits(0xBE2AAAABu)));
+    S = fma2(p, mul2(r2, r), r);
+    f2 c = fma2(splat(fbits(0xB493F27Eu)), r2, splat(fbits(0x37D00D01u)));
+    c = fma2(c, r2, splat(fbits(0xBAB60B61u)));
+    c = fma2(c, r2, splat(fbits(0x3D2AAAABu)));
+    c = fma2(c, r2, splat(-0.5f));
+    C = fma2(c, r2, splat(1.0f));
+    qa = __float_as_uint(lo(nb));
+    qb = __float_as_uint(hi(nb));
+}
+
+// sin of two arguments: one select and one sign flip per element.
+__device__ __forceinline__ f2 sin2(f2 x)
+{
+    f2 S, C; uint32_t qa, qb;
+    sincos_poly2(x, S, C, qa, qb);
+    const float sa = (qa & 1u) ? lo(C) : lo(S);
+    const float sb = (qb & 1u) ? hi(C) : hi(S);
+    return pk(__uint_as_float(__float_as_uint(sa) ^ ((qa << 30) & 0x80000000u)),
+              __uint_as_float(__float_as_uint(sb) ^ ((qb << 30) & 0x80000000u)));
+}
+
+// cos of two arguments.
+__device__ __forceinline__ f2 cos2(f2 x)
+{
+    f2 S, C; uint32_t qa, qb;
+    sincos_poly2(x, S, C, qa, qb);
+    const float ca = (qa & 1u) ? lo(S) : lo(C);
+    const float cb = (qb & 1u) ? hi(S) : hi(C);
+    return pk(__uint_as_float(__float_as_uint(ca) ^ (((qa + 1u) << 30) & 0x80000000u)),
+              __uint_as_float(__float_as_uint(cb) ^ (((qb + 1u) << 30) & 0x80000000u)));
+}
+
+// sin and cos of two arguments, and the negated sin (one more xor per element).
+__device__ __forceinline__ void sincos2_full(f2 x, f2 &sn, f2 &nsn, f2 &cs)
+{
+    f2 S, C; uint32_t qa, qb;
+    sincos_poly2(x, S, C, qa, qb);
+    const bool oa = qa & 1u, ob = qb & 1u;
+    const uint32_t sa = __float_as_uint(oa ? lo(C) : lo(S)) ^ ((qa << 30) & 0x80000000u);
+    const uint32_t sb = __float_as_uint(ob ? hi(C) : hi(S)) ^ ((qb << 30) & 0x80000000u);
+    const float ca = oa ? lo(S) : lo(C), cb = ob ? hi(S) : hi(C);
+    sn = pk(__uint_as_float(sa), __uint_as_float(sb));
+    nsn = pk(__uint_as_float(sa ^ 0x80000000u), __uint_as_float(sb ^ 0x80000000u));
+    cs = pk(__uint_as_float(__float_as_uint(ca) ^ (((qa + 1u) << 30) & 0x80000000u)),
+            __uint_as_float(__float_as_uint(cb) ^ (((qb + 1u) << 30) & 0x80000000u)));
+}
+
+__device__ __forceinline__ f2 neg2(f2 a) { return pk(-lo(a), -hi(a)); }
+
 __device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
+// Correctly rounded reciprocals of two denominators that lie in a range for which the library's
+// arithmetic self-check has verified, value by value, that one Newton step from the hardware
+// approximation equals the IEEE reciprocal.  nd = -d.
+__device__ __forceinline__ f2 rcp2_refined(f2 d, f2 nd)
+{
+    const f2 y0 = pk(rcp_approx(lo(d)), rcp_approx(hi(d)));
+    return fma2(y0, fma2(nd, y0, splat(1.0f)), y0);
+}
+
+// IEEE quotients num/d given y = RN(1/d) and nd = -d: estimate, exact residual, correction.  Exact when the
+// numerator's exponent lies in [2^-63, 2^65) (see exponent_guard) or the numerator needs no guard.
+__device__ __forceinline__ f2 div2_refined(f2 num, f2 y, f2 nd)
+{
+    const f2 q0 = mul2(num, y);
+    return fma2(fma2(nd, q0, num), y, q0);
+}
+
+// Accumulates into bit 30 of `acc` whether either half of v has its two top exponent bits equal, i.e.
+// lies outside [2^-63, 2^65) (zero, tiny, huge, infinite or NaN).
+__device__ __forceinline__ void exponent_guard(f2 v, uint32_t &acc)
+{
+    const uint32_t a = __float_as_uint(lo(v)), b = __float_as_uint(hi(v));
+    acc |= ~(a ^ (a << 1)) | ~(b ^ (b << 1));
+}
 
 // exp of two arguments already inside [-87, 88] (same operations as exp_core, two at a time).
 __device__ __forceinline__ f2 exp2_core(f2 y)
