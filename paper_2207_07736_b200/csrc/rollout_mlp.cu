@@ -121,7 +121,10 @@ __device__ __forceinline__ int sample_pair(f2 l, uint32_t w)
     return (thr < lo(e)) ? 0 : 1;
 }
 
-constexpr int kMlp2Threads = 128;  // 4 warps x 64 envs
+#ifndef MLP_THREADS
+#define MLP_THREADS 128
+#endif
+constexpr int kMlp2Threads = MLP_THREADS;  // warps of 64 envs each
 
 __global__ void __launch_bounds__(kMlp2Threads, MLP_MINBLOCKS)
 rollout_cartpole_mlp_kernel(const __grid_constant__ S4Args a)
