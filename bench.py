@@ -144,6 +144,8 @@ def run_reference(args, w):
     if rank != 0:
         return 0
     per_step_budget = max(0.2, min(5.0, 60.0 / max(1, args.steps + args.warmup)))
+    if args.cpu_seconds != 10.0:                                    # explicit budget per step
+        per_step_budget = args.cpu_seconds
     for _ in range(args.warmup):
         oracle_rate(w, per_step_budget, compute_factor=args.compute_factor)
     rates, sample = [], ""

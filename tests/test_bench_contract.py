@@ -1,0 +1,41 @@
+"""The bench's reference arm and its roofline arithmetic (CPU only; the GPU arm is exercised on the B200)."""
+import json
+import os
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+import bench  # noqa: E402
+from paper_2207_07736_b200 import inputs  # noqa: E402
+
+
+def test_algorithmic_bytes_and_flops():
+    w2, w5 = inputs.WORKLOADS["cfg2"], inputs.WORKLOADS["cfg5_S4096"]
+    assert bench.algorithmic_bytes_per_env_step(w2, 1) == 22 + 48
+    assert abs(bench.algorithmic_bytes_per_env_step(w2, 1000) - 22.048) < 1e-9
+    assert bench.algorithmic_bytes_per_env_step(w5, 1) == 8 * 4096 + 16          # no trajectory for the synthetic config
+    assert bench.algorithmic_bytes_per_env_step(w5, 4) == (8 * 4096 + 16) / 4
+    assert bench.nominal_flops_per_env_step(w2) == (27, 52)
+    assert bench.nominal_flops_per_env_step(inputs.WORKLOADS["cfg3"]) == (27 + 9094, 52 + 12205)
+    assert bench.nominal_flops_per_env_step(w5) == (7 * 4096, 24 * 4096)
+
+
+def test_reference_arm_prints_the_contract_line():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "2", "--warmup", "3",
+                          "--cpu-seconds", "0.05"], capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["metric"] == "env_steps_per_sec" and line["unit"] == "env-steps/s"
+    assert line["higher_is_better"] is True and line["steps"] == 2 and line["warmup"] == 3 and line["value"] > 1e5
+    assert line["config"]["workload"] == "cfg2" and line["vs_baseline"] is None
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1 and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"] == {"value": line["value"], "unit": "env-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+
+
+def test_reference_arm_other_ranks_do_nothing():
+    env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1"],
+                         capture_output=True, text=True, timeout=60, cwd=ROOT, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
