@@ -260,6 +260,37 @@ def test_cartpole_window_path_edge_cases():
         run_pair(oracle.CARTPOLE, 515, 40, K, seed=21, pre=pre)
 
 
+def test_outputs_stay_inside_their_buffers():
+    """Canary words around every output buffer (the pool has no memory checker): ragged env counts, every
+    kernel, K that does not divide T; nothing outside [T,N,...] may be written."""
+    torch = torch_cuda()
+    PAD = 4096
+    cases = [(oracle.CARTPOLE, 4, 1003, 37, 8, None), (oracle.CARTPOLE, 4, 65, 19, 19, inputs.mlp_params(2)),
+             (oracle.ACROBOT, 4, 197, 23, 7, None), (oracle.ACROBOT, 4, 130, 5, 2, None),
+             (oracle.SYNTH, 4, 999, 9, 4, None), (oracle.SYNTH, 64, 33, 9, 9, None), (oracle.SYNTH, 2048, 3, 5, 2, None)]
+    for kind, S, n, T, K, params in cases:
+        sizes = {"obs": T * n * S * 4, "act": T * n, "rew": T * n * 4, "done": T * n}
+        bufs, views = {}, {}
+        for name, nbytes in sizes.items():
+            padded = (nbytes + 15) // 16 * 16
+            b = torch.full((PAD + padded + PAD,), 0xA5, dtype=torch.uint8, device="cuda")
+            bufs[name] = (b, nbytes)
+            views[name] = b[PAD:PAD + nbytes]
+        sim = binding.Sim(kind, n, S, 4)
+        d_params = None if params is None else torch.from_numpy(params).cuda()
+        binding.sim_rollout(sim.h, T, K, d_params, views["obs"], views["act"], views["rew"], views["done"])
+        state_before = sim.state().clone()
+        torch.cuda.synchronize()
+        for name, (b, nbytes) in bufs.items():
+            assert bool((b[:PAD] == 0xA5).all()) and bool((b[PAD + nbytes:] == 0xA5).all()), (kind, S, name)
+        done = views["done"].view(T, n)
+        assert int(done.max()) <= 1
+        # and the handle's own buffers: a second handle created right after must not be disturbed by the first
+        other = binding.Sim(kind, n, S, 4)
+        ref = other.rollout(T, K, d_params)
+        assert torch.equal(ref["done"], done) and torch.equal(other.state(), state_before)
+
+
 def test_argument_errors_with_live_handle():
     torch = torch_cuda()
     sim = binding.Sim(oracle.ACROBOT, 16)
