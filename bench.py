@@ -194,6 +194,14 @@ def run_gpu(args, w):
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the CPU oracle")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    if not binding.LIB_PATH.exists():                               # normally built in-tree beforehand
+        if local_rank == 0:
+            from paper_2207_07736_b200 import build as _build
+            _build.build()
+        else:
+            t_wait = time.time()
+            while not binding.LIB_PATH.exists() and time.time() - t_wait < 600:
+                time.sleep(1.0)
     dist = shard.init_process_group("nccl")
     hbm_peak, sm_max_mhz, peak_kind = measured_peaks()
 
