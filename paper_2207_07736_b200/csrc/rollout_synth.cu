@@ -13,10 +13,20 @@
 #include "sim_internal.h"
 #include "sim_envs.cuh"
 
+#ifndef SYNTH_E_LONG_CAP
+#define SYNTH_E_LONG_CAP 64
+#endif
+
 namespace simk {
 
-template <int S> struct SynthShape {
-    static constexpr int E = S <= 128 ? 4 : (S <= 512 ? S / 32 : 16);   // floats per thread
+// Floats per thread.  Short launches (a stream over the state matrix) want many small chunks: coalesced
+// float4 accesses and many threads in flight.  Long launches want long chunks: fewer shuffles, halo
+// exchanges and barriers per element and more independent pairs per thread.
+constexpr int synth_chunk_short(int S) { return S <= 128 ? 4 : (S <= 512 ? S / 32 : 16); }
+constexpr int synth_chunk_long(int S) { return S < SYNTH_E_LONG_CAP ? S : SYNTH_E_LONG_CAP; }
+
+template <int S, int E_> struct SynthShape {
+    static constexpr int E = E_;                                        // floats per thread
     static constexpr int H = E / 2;                                     // packed pairs per thread
     static constexpr int L = S / E;                                     // threads per env
     static constexpr int WARPS = L > 32 ? L / 32 : 1;                   // warps per env when L > 32
@@ -29,11 +39,11 @@ template <int W> struct SynthExchange { float halo[2][W]; float sum[W]; };   // 
 
 // K steps of one chunk held in registers.  P[j] = (x_j, x_{j+H}).  All threads of a CTA call this
 // together (it contains CTA barriers when an env spans several warps).
-template <int S>
-__device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[SynthShape<S>::H], uint32_t &len, uint32_t &rc,
-                                            uint32_t i, bool valid, uint32_t sub, SynthExchange<SynthShape<S>::WARPS> &xc)
+template <int S, int EE>
+__device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[EE / 2], uint32_t &len, uint32_t &rc,
+                                            uint32_t i, bool valid, uint32_t sub, SynthExchange<SynthShape<S, EE>::WARPS> &xc)
 {
-    using Sh = SynthShape<S>;
+    using Sh = SynthShape<S, EE>;
     constexpr int E = Sh::E, H = Sh::H, L = Sh::L, W = Sh::WARPS;
     constexpr int LS = L < 32 ? L : 32;                 // lanes of one env inside a warp
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -140,11 +150,11 @@ __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[SynthSha
     }
 }
 
-template <int S>
-__device__ __forceinline__ void synth_store(const SynthArgs &a, const f2 (&P)[SynthShape<S>::H], uint32_t len, uint32_t rc,
+template <int S, int EE>
+__device__ __forceinline__ void synth_store(const SynthArgs &a, const f2 (&P)[EE / 2], uint32_t len, uint32_t rc,
                                             uint32_t i, uint32_t sub)
 {
-    constexpr int E = SynthShape<S>::E, H = SynthShape<S>::H;
+    constexpr int E = EE, H = EE / 2;
     float xo[E];
 #pragma unroll
     for (int j = 0; j < H; ++j) { xo[j] = lo(P[j]); xo[j + H] = hi(P[j]); }
@@ -162,11 +172,11 @@ __device__ __forceinline__ void synth_store(const SynthArgs &a, const f2 (&P)[Sy
 // One tile (THREADS chunks) per CTA; each thread loads its chunk straight into registers.  (A persistent
 // variant with a cp.async ring of shared-memory stages was measured for K = 1 and was slower: at K = 1
 // the launch is bound by instruction issue per tile, not by bytes in flight.)
-template <int S>
-__global__ void __launch_bounds__(SynthShape<S>::THREADS)
+template <int S, int EE>
+__global__ void __launch_bounds__(SynthShape<S, EE>::THREADS)
 rollout_synth_kernel(const __grid_constant__ SynthArgs a)
 {
-    using Sh = SynthShape<S>;
+    using Sh = SynthShape<S, EE>;
     constexpr int E = Sh::E, H = Sh::H, L = Sh::L;
     __shared__ SynthExchange<Sh::WARPS> xc;
     const uint32_t tid = threadIdx.x;
@@ -187,16 +197,25 @@ rollout_synth_kernel(const __grid_constant__ SynthArgs a)
         for (int j = 0; j < H; ++j) P[j] = pk(xin[j], xin[j + H]);
     }
     uint32_t len = a.ep_len[i], rc = a.reset_count[i];
-    synth_steps<S>(a, P, len, rc, i, valid, sub, xc);
-    if (valid) synth_store<S>(a, P, len, rc, i, sub);
+    synth_steps<S, EE>(a, P, len, rc, i, valid, sub, xc);
+    if (valid) synth_store<S, EE>(a, P, len, rc, i, sub);
 }
+
+template <int S, int EE>
+static cudaError_t launch_synth_e(const SynthArgs &a, cudaStream_t st)
+{
+    using Sh = SynthShape<S, EE>;
+    const uint32_t ntiles = (a.n + Sh::ENVS_PER_CTA - 1u) / Sh::ENVS_PER_CTA;
+    return launch_overlapped(a.K <= kOverlapMaxK, rollout_synth_kernel<S, EE>, dim3(ntiles), dim3(Sh::THREADS), 0, st, a);
+}
+
+constexpr int kSynthLongK = 3;     // launches of at least this many steps use the long-chunk shape
 
 template <int S>
 static cudaError_t launch_synth_t(const SynthArgs &a, cudaStream_t st)
 {
-    using Sh = SynthShape<S>;
-    const uint32_t ntiles = (a.n + Sh::ENVS_PER_CTA - 1u) / Sh::ENVS_PER_CTA;
-    return launch_overlapped(a.K <= kOverlapMaxK, rollout_synth_kernel<S>, dim3(ntiles), dim3(Sh::THREADS), 0, st, a);
+    if (a.K >= kSynthLongK) return launch_synth_e<S, synth_chunk_long(S)>(a, st);
+    return launch_synth_e<S, synth_chunk_short(S)>(a, st);
 }
 
 cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st)
