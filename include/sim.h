@@ -132,6 +132,13 @@ int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t *d_reset
  *   any live handle (it provides the stream). */
 int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits);
 
+/* sim_acrobot_observation -- the six-value observation an RL consumer of Acrobot usually wants,
+ * (cos theta1, sin theta1, cos theta2, sin theta2, omega1, omega2), from raw 4-float states (the
+ * trajectory's out_obs rows, or sim_get_state): d_state [M,4] fp32 -> d_obs6 [M,6] fp32, both device
+ * pointers, 16- and 8-byte aligned.  Uses the library's specified sin/cos, so it is reproducible bit for
+ * bit.  (The paper's simulators expose raw state only; this is a convenience on top of the path.) */
+int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, float *d_obs6);
+
 /* sim_selfcheck_division -- numerical self-check of the divisions inside the fused kernels (the paper
  * has no counterpart; it exists so a test can prove the kernels' arithmetic on the device they run
  * on).  The fused CartPole and Acrobot kernels divide by well-conditioned denominators with a refined

@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
         L.oracle_acrobot_dsdt.restype = None
         L.oracle_acrobot_step.argtypes = [f32p, C.c_int, f32p]
         L.oracle_acrobot_step.restype = C.c_int
+        L.oracle_acrobot_observation.argtypes = [f32p, f32p]
+        L.oracle_acrobot_observation.restype = None
         L.oracle_synth_step.argtypes = [f32p, C.c_int, C.c_int, f32p, f32p]
         L.oracle_synth_step.restype = C.c_int
         L.oracle_pairwise_sum.argtypes = [f32p, C.c_int]
@@ -190,6 +192,13 @@ def acrobot_step(s, act):
     out = np.zeros(4, dtype=np.float32)
     goal = lib().oracle_acrobot_step(_fp(s), int(act), _fp(out))
     return out, int(goal)
+
+
+def acrobot_observation(s):
+    s = _f32(s)
+    out = np.zeros(6, dtype=np.float32)
+    lib().oracle_acrobot_observation(_fp(s), _fp(out))
+    return out
 
 
 def synth_step(x, act):

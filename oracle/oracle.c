@@ -310,6 +310,15 @@ ORACLE_API int oracle_acrobot_step(const float s[4], int act, float out[4])
     return g > 1.0f;
 }
 
+/* Gym-style six-value observation of an Acrobot state: (cos t1, sin t1, cos t2, sin t2, w1, w2). */
+ORACLE_API void oracle_acrobot_observation(const float s[4], float out[6])
+{
+    oracle_sincos_s(s[0], &out[1], &out[0]);
+    oracle_sincos_s(s[1], &out[3], &out[2]);
+    out[4] = s[2];
+    out[5] = s[3];
+}
+
 /* ------------------------------------------------------------------------------------
  * Synthetic S-float simulator (the paper's "state factor" knob of Section 4.2, with the
  * per-element update the benchmark spec gives).  Jacobi update: every right-hand side

@@ -33,6 +33,7 @@ SIGNATURES = {
     "sim_get_counters": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_uint64)]),
     "sim_set_counters": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]),
     "sim_policy_logits": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
+    "sim_acrobot_observation": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "sim_selfcheck_division": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_uint64)]),
     "sim_rollout_noalloc": (C.c_int, [C.c_int, C.c_int64, C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -142,6 +143,10 @@ def sim_set_counters(h, d_ep_len, d_reset_count, t):
 
 def sim_policy_logits(h, d_obs, M, d_params, d_logits):
     _check(lib().sim_policy_logits(h, _ptr(d_obs), M, _ptr(d_params), _ptr(d_logits)), h)
+
+
+def sim_acrobot_observation(h, d_state, M, d_obs6):
+    _check(lib().sim_acrobot_observation(h, _ptr(d_state), M, _ptr(d_obs6)), h)
 
 
 def sim_selfcheck_division(h, nums_per_den):

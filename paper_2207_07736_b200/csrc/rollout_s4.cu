@@ -122,6 +122,31 @@ reset_synth_kernel(float4 *state, uint32_t *ep_len, uint32_t *reset_count, uint3
     if (j == 0) { ep_len[i] = 0u; reset_count[i] = 0u; }
 }
 
+// Gym-style six-value Acrobot observation (cos t1, sin t1, cos t2, sin t2, w1, w2) of M states.
+__global__ void __launch_bounds__(256)
+acrobot_observation_kernel(const float4 *__restrict__ state, int64_t M, float *__restrict__ obs6)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M) return;
+    const float4 s = state[i];
+    float s1, c1, s2, c2;
+    sincos_s(s.x, s1, c1);
+    sincos_s(s.y, s2, c2);
+    float2 *o = reinterpret_cast<float2 *>(obs6 + i * 6);       // rows of 24 bytes: 8-byte aligned
+    o[0] = make_float2(c1, s1);
+    o[1] = make_float2(c2, s2);
+    o[2] = make_float2(s.z, s.w);
+}
+
+cudaError_t launch_acrobot_observation(const float *state, int64_t M, float *obs6, cudaStream_t st)
+{
+    if (M <= 0) return cudaSuccess;
+    const int64_t blocks = (M + 255) / 256;
+    if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
+    acrobot_observation_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(state), M, obs6);
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------------------------

@@ -350,3 +350,11 @@ SIM_API int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_misma
     *h_mismatches = (uint64_t)h;
     return SIM_OK;
 }
+
+SIM_API int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, float *d_obs6)
+{
+    if (!s || !d_state || !d_obs6 || M < 0) return SIM_EINVAL;
+    CU(s, launch_acrobot_observation(d_state, M, d_obs6, s->stream));
+    if (M > 0) s->launches += 1;
+    return SIM_OK;
+}

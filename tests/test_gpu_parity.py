@@ -291,6 +291,20 @@ def test_outputs_stay_inside_their_buffers():
         assert torch.equal(ref["done"], done) and torch.equal(other.state(), state_before)
 
 
+def test_acrobot_six_value_observation():
+    torch = torch_cuda()
+    sim = binding.Sim(oracle.ACROBOT, 300, 4, 3)
+    out = sim.rollout(40, 40)
+    states = out["obs"].reshape(-1, 4).contiguous()
+    obs6 = torch.empty((states.shape[0], 6), dtype=torch.float32, device="cuda")
+    binding.sim_acrobot_observation(sim.h, states, states.shape[0], obs6)
+    got = to_np(obs6)
+    st = to_np(states)
+    for i in range(0, st.shape[0], 97):
+        assert_same_bits(got[i], oracle.acrobot_observation(st[i]), "obs6 row %d" % i)
+    assert float((obs6[:, 0] ** 2 + obs6[:, 1] ** 2 - 1).abs().max()) < 1e-6
+
+
 def test_argument_errors_with_live_handle():
     torch = torch_cuda()
     sim = binding.Sim(oracle.ACROBOT, 16)

@@ -138,3 +138,13 @@ def test_time_limit_and_reward_through_rollout():
     # most random-torque episodes run into the limit
     first_done = np.array([np.flatnonzero(done[:, e])[0] for e in range(sim.n)])
     assert np.mean(first_done == 499) > 0.9
+
+
+def test_six_value_observation():
+    rng = np.random.default_rng(9)
+    for _ in range(200):
+        s = (rng.uniform(-1, 1, 4) * np.array([math.pi, math.pi, 12, 28])).astype(np.float32)
+        o = oracle.acrobot_observation(s).astype(np.float64)
+        want = [math.cos(float(s[0])), math.sin(float(s[0])), math.cos(float(s[1])), math.sin(float(s[1])), float(s[2]), float(s[3])]
+        assert np.abs(o - want).max() < 3e-7
+    assert np.array_equal(oracle.acrobot_observation([0, 0, 1.5, -2.5]), np.array([1, 0, 1, 0, 1.5, -2.5], np.float32))
