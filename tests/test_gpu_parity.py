@@ -261,7 +261,7 @@ def test_cartpole_window_path_edge_cases():
 
 
 def test_outputs_stay_inside_their_buffers():
-    """Canary words around every output buffer (the pool has no memory checker): ragged env counts, every
+    """Canary words around every output buffer (no memory checker runs on these kernels): ragged env counts, every
     kernel, K that does not divide T; nothing outside [T,N,...] may be written."""
     torch = torch_cuda()
     PAD = 4096
