@@ -305,6 +305,36 @@ def test_acrobot_six_value_observation():
     assert float((obs6[:, 0] ** 2 + obs6[:, 1] ** 2 - 1).abs().max()) < 1e-6
 
 
+def test_random_shapes_against_the_oracle():
+    """Forty seeded random (env kind, S, N, T, K, C, seed, policy) combinations, including N = 1, K > T and
+    rollouts split in two calls."""
+    torch = torch_cuda()
+    rng = np.random.default_rng(2024)
+    p_mlp = inputs.mlp_params(5, 0.3)
+    for case in range(40):
+        kind = int(rng.integers(0, 3))
+        S = int(2 ** rng.integers(2, 13)) if kind == oracle.SYNTH else 4
+        n = 1 if case % 10 == 0 else int(rng.integers(1, 700 if S <= 256 else 12))
+        T = int(rng.integers(1, 60))
+        K = int(rng.integers(1, T + 4))
+        C = int(rng.choice([1, 1, 2, 3]))
+        seed = int(rng.integers(0, 2 ** 63))
+        params = p_mlp if (kind == oracle.CARTPOLE and case % 3 == 0) else None
+        sim = binding.Sim(kind, n, S, seed, compute_factor=C)
+        orc = oracle.OracleSim(kind, n, S, seed, compute_factor=C)
+        d_params = None if params is None else torch.from_numpy(params).cuda()
+        T1 = int(rng.integers(0, T + 1))
+        outs = []
+        if T1 > 0:
+            outs.append(sim.rollout(T1, K, d_params))
+        if T - T1 > 0:
+            outs.append(sim.rollout(T - T1, max(1, K - 1), d_params))
+        torch.cuda.synchronize()
+        ref = orc.rollout(T, policy_params=params)
+        out = {k: torch.cat([o[k] for o in outs]) for k in ("obs", "act", "rew", "done")}
+        compare_rollout(out, sim, ref, orc, what="case %d kind %d S %d n %d T %d K %d C %d" % (case, kind, S, n, T, K, C))
+
+
 def test_argument_errors_with_live_handle():
     torch = torch_cuda()
     sim = binding.Sim(oracle.ACROBOT, 16)
