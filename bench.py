@@ -363,9 +363,10 @@ def run_grid(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py --grid needs a CUDA device")
     T, ks = 64, (1, 8, 64)
-    for S in (4, 64, 512, 4096):
-        n = (128 << 20) // S                                   # 512 MiB of state: streams from HBM at K = 1
-        for C in (1, 4, 16, 64):
+    points = [(S, (128 << 20) // S, C) for S in (4, 64, 512, 4096) for C in (1, 4, 16, 64)]   # 512 MiB of state: streams from HBM at K = 1
+    points += [(S, (32 << 20) // S, 1) for S in (4, 64, 512, 4096)]                            # the N axis: a quarter of the envs
+    for S, n, C in points:
+        if True:
             sim = binding.Sim(inputs.SYNTH, n, S, 0, compute_factor=C)
             w = dataclasses.replace(inputs.WORKLOADS["cfg5_S%d" % S], n_envs=n, T=T)
             row = {"grid": "simulator_complexity", "S": S, "C": C, "n_envs": n, "T": T, "k": {}}
