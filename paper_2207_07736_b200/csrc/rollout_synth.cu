@@ -13,16 +13,20 @@
 #include "sim_internal.h"
 #include "sim_envs.cuh"
 
+#ifndef SYNTH_E_SHORT
+#define SYNTH_E_SHORT 16
+#endif
 #ifndef SYNTH_E_LONG_CAP
 #define SYNTH_E_LONG_CAP 64
 #endif
 
 namespace simk {
 
-// Floats per thread.  Short launches (a stream over the state matrix) want many small chunks: coalesced
-// float4 accesses and many threads in flight.  Long launches want long chunks: fewer shuffles, halo
-// exchanges and barriers per element and more independent pairs per thread.
-constexpr int synth_chunk_short(int S) { return S <= 128 ? 4 : (S <= 512 ? S / 32 : 16); }
+// Floats per thread.  Long launches want long chunks (64): few shuffles, halo exchanges and barriers per
+// element and many independent pairs per thread.  Short launches (a stream over the state matrix) want
+// more threads in flight and do best with 16 (measured at K = 1: 4 -> 3.3e11, 8 -> 4.9e11, 16 -> 5.7e11
+// element-steps/s for S = 16..128; the per-thread overhead of a tile is what a short launch pays for).
+constexpr int synth_chunk_short(int S) { return S < SYNTH_E_SHORT ? S : SYNTH_E_SHORT; }
 constexpr int synth_chunk_long(int S) { return S < SYNTH_E_LONG_CAP ? S : SYNTH_E_LONG_CAP; }
 
 template <int S, int E_> struct SynthShape {
