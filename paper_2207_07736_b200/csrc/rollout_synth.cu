@@ -43,7 +43,7 @@ template <int W> struct SynthExchange { float halo[2][W]; float sum[W]; };   // 
 
 // K steps of one chunk held in registers.  P[j] = (x_j, x_{j+H}).  All threads of a CTA call this
 // together (it contains CTA barriers when an env spans several warps).
-template <int S, int EE>
+template <int S, int EE, bool LEAN>
 __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[EE / 2], uint32_t &len, uint32_t &rc,
                                             uint32_t i, bool valid, uint32_t sub, SynthExchange<SynthShape<S, EE>::WARPS> &xc)
 {
@@ -58,14 +58,14 @@ __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[EE / 2],
     const int nblk = (a.phase + a.K + 3) >> 2;
     for (int b = 0; b < nblk; ++b) {
         uint4 blk = make_uint4(0u, 0u, 0u, 0u);
-        if (!a.actions) blk = philox(env, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
-#pragma unroll 1
+        if (LEAN || !a.actions) blk = philox(env, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
+#pragma unroll(EE <= 8 ? 4 : 1)
         for (int j4 = 0; j4 < 4; ++j4) {
             const int k = 4 * b + j4 - a.phase;
             if (k < 0 || k >= a.K) continue;
             const uint32_t w = j4 == 0 ? blk.x : j4 == 1 ? blk.y : j4 == 2 ? blk.z : blk.w;
 
-            if (a.out_obs && valid) {
+            if (!LEAN && a.out_obs && valid) {
                 float *dst = a.out_obs + row * S + (size_t)sub * E;
                 float xo[E];
 #pragma unroll
@@ -75,7 +75,7 @@ __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[EE / 2],
                     __stcs(reinterpret_cast<float4 *>(dst + 4 * v), make_float4(xo[4 * v], xo[4 * v + 1], xo[4 * v + 2], xo[4 * v + 3]));
             }
 
-            const int act = a.actions ? (a.actions[i] != 0) : (int)(w >> 31);
+            const int act = (!LEAN && a.actions) ? (a.actions[i] != 0) : (int)(w >> 31);
             const f2 c = splat(__fmul_rn(fbits(0x3A83126Fu), act ? 1.0f : -1.0f));
 
             // compute factor: C Jacobi iterations under one action; squares and the done test use the last one
@@ -131,7 +131,7 @@ __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[EE / 2],
             const bool done = __fmul_rn(sum, 1.0f / (float)S) > 4.0f;
             len += 1u;
 
-            if (leader) {
+            if (!LEAN && leader) {
                 if (a.out_act) __stcs(&a.out_act[row], (int8_t)act);
                 if (a.out_rew) __stcs(&a.out_rew[row], 1.0f);
                 if (a.out_done) __stcs(&a.out_done[row], (uint8_t)done);
@@ -176,7 +176,9 @@ __device__ __forceinline__ void synth_store(const SynthArgs &a, const f2 (&P)[EE
 // One tile (THREADS chunks) per CTA; each thread loads its chunk straight into registers.  (A persistent
 // variant with a cp.async ring of shared-memory stages was measured for K = 1 and was slower: at K = 1
 // the launch is bound by instruction issue per tile, not by bytes in flight.)
-template <int S, int EE>
+// LEAN: no trajectory output and random actions (the timed configuration of the synthetic workload); the
+// per-step checks for optional outputs and given actions are compiled out.
+template <int S, int EE, bool LEAN>
 __global__ void __launch_bounds__(SynthShape<S, EE>::THREADS)
 rollout_synth_kernel(const __grid_constant__ SynthArgs a)
 {
@@ -201,7 +203,7 @@ rollout_synth_kernel(const __grid_constant__ SynthArgs a)
         for (int j = 0; j < H; ++j) P[j] = pk(xin[j], xin[j + H]);
     }
     uint32_t len = a.ep_len[i], rc = a.reset_count[i];
-    synth_steps<S, EE>(a, P, len, rc, i, valid, sub, xc);
+    synth_steps<S, EE, LEAN>(a, P, len, rc, i, valid, sub, xc);
     if (valid) synth_store<S, EE>(a, P, len, rc, i, sub);
 }
 
@@ -210,7 +212,9 @@ static cudaError_t launch_synth_e(const SynthArgs &a, cudaStream_t st)
 {
     using Sh = SynthShape<S, EE>;
     const uint32_t ntiles = (a.n + Sh::ENVS_PER_CTA - 1u) / Sh::ENVS_PER_CTA;
-    return launch_overlapped(a.K <= kOverlapMaxK, rollout_synth_kernel<S, EE>, dim3(ntiles), dim3(Sh::THREADS), 0, st, a);
+    const bool lean = !a.out_obs && !a.out_act && !a.out_rew && !a.out_done && !a.actions;
+    if (lean) return launch_overlapped(a.K <= kOverlapMaxK, rollout_synth_kernel<S, EE, true>, dim3(ntiles), dim3(Sh::THREADS), 0, st, a);
+    return launch_overlapped(a.K <= kOverlapMaxK, rollout_synth_kernel<S, EE, false>, dim3(ntiles), dim3(Sh::THREADS), 0, st, a);
 }
 
 constexpr int kSynthLongK = 3;     // launches of at least this many steps use the long-chunk shape
