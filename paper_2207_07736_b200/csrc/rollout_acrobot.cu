@@ -80,10 +80,11 @@ __global__ void __launch_bounds__(kAcroThreads)
 rollout_acrobot_x2_kernel(const __grid_constant__ S4Args a)
 {
     const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t base = (blockIdx.x * (kAcroThreads / 32) + (threadIdx.x >> 5)) * 64u;
-    if (base >= a.n) return;
+    const uint64_t base64 = ((uint64_t)blockIdx.x * (kAcroThreads / 32) + (threadIdx.x >> 5)) * 64u;   // may exceed 2^32 near the largest N
+    if (base64 >= a.n) return;
+    const uint32_t base = (uint32_t)base64;
     uint32_t ia = base + lane, ib = base + 32u + lane;
-    const bool va = ia < a.n, vb = ib < a.n;            // tail envs: computed on a clamped index, never stored
+    const bool va = base64 + lane < a.n, vb = base64 + 32u + lane < a.n;   // tail envs: computed on a clamped index, never stored
     if (!va) ia = a.n - 1u;
     if (!vb) ib = a.n - 1u;
     const uint32_t env_a = a.env_offset + ia, env_b = a.env_offset + ib;

@@ -45,8 +45,9 @@ template <int ENV, int POLICY>
 __global__ void __launch_bounds__(kS4Threads)
 rollout_s4_kernel(const __grid_constant__ S4Args a)
 {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= a.n) return;
+    const uint64_t i64 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i64 >= a.n) return;
+    const uint32_t i = (uint32_t)i64;
     const uint32_t env = a.env_offset + i;
     pdl_wait();
     pdl_release();
@@ -101,8 +102,9 @@ template <int ENV>
 __global__ void __launch_bounds__(256)
 reset_s4_kernel(float4 *state, uint32_t *ep_len, uint32_t *reset_count, uint32_t n, uint32_t env_offset, const __grid_constant__ RoundKeys rk)
 {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
+    const uint64_t i64 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i64 >= n) return;
+    const uint32_t i = (uint32_t)i64;
     state[i] = draw_state4<ENV>(env_offset + i, 0u, 0u, rk);
     ep_len[i] = 0u;
     reset_count[i] = 0u;

@@ -187,9 +187,9 @@ rollout_synth_kernel(const __grid_constant__ SynthArgs a)
     __shared__ SynthExchange<Sh::WARPS> xc;
     const uint32_t tid = threadIdx.x;
     const uint32_t sub = tid % L;
-    uint32_t i = blockIdx.x * (uint32_t)Sh::ENVS_PER_CTA + tid / L;
-    const bool valid = i < a.n;                         // tail threads compute on env n-1 and store nothing
-    if (!valid) i = a.n - 1u;
+    const uint64_t i64 = (uint64_t)blockIdx.x * Sh::ENVS_PER_CTA + tid / L;
+    const bool valid = i64 < a.n;                       // tail threads compute on env n-1 and store nothing
+    uint32_t i = valid ? (uint32_t)i64 : a.n - 1u;
     pdl_wait();
     pdl_release();
 
