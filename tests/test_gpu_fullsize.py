@@ -56,3 +56,21 @@ def test_cfg4_acrobot_full():
 @pytest.mark.parametrize("S,K,ns", [(4, 256, 4000), (64, 64, 500), (512, 16, 64), (4096, 256, 10), (4096, 1, 10)])
 def test_cfg5_synth_full(S, K, ns):
     sampled_check("cfg5_S%d" % S, K, ns)
+
+
+@pytest.mark.parametrize("kind", [oracle.CARTPOLE, oracle.ACROBOT])
+def test_very_large_ragged_batch(kind):
+    """Fifty million envs with a ragged tail: 64-bit trajectory indexing and the last partial warp."""
+    torch = torch_cuda()
+    n, T = 50_000_017, 9
+    sim = binding.Sim(kind, n, 4, 7)
+    out = sim.rollout(T, 9, want=("obs", "done"))
+    torch.cuda.synchronize()
+    ids = np.concatenate([inputs.sample_env_ids(1, n, 40), np.arange(n - 70, n, dtype=np.uint32)])
+    ids = np.unique(ids)
+    orc = oracle.OracleSim(kind, state_dim=4, seed=7, env_ids=ids)
+    ref = orc.rollout(T, want=("obs", "done"))
+    sel = torch.from_numpy(ids.astype(np.int64)).cuda()
+    assert_same_bits(to_np(out["obs"][:, sel]), ref["obs"], "obs")
+    assert_same_bits(to_np(out["done"][:, sel]), ref["done"], "done")
+    assert_same_bits(to_np(sim.state()[sel]), orc.state, "state")
