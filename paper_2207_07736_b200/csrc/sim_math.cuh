@@ -129,52 +129,6 @@ __device__ __forceinline__ f2 sub2(f2 a, f2 b) { f2 r; asm("sub.rn.f32x2 %0, %1,
 __device__ __forceinline__ f2 mul2(f2 a, f2 b) { f2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
 
 
-// Quadrant fix-up of one (S, C) polynomial pair: q = k mod 4 in the low bits.
-__device__ __forceinline__ void quadrant_fix(uint32_t q, float S, float C, float &sn, float &cs)
-{
-    const bool odd = q & 1u;
-    const float a = odd ? C : S;
-    const float b = odd ? S : C;
-    sn = __uint_as_float(__float_as_uint(a) ^ ((q & 2u) << 30));
-    cs = __uint_as_float(__float_as_uint(b) ^ (((q + 1u) & 2u) << 30));
-}
-
-// sin and cos of two arguments at once.  `converged_mask` names the lanes that execute this call
-// together (all of them must): when no lane of the warp leaves the first quadrant's neighbourhood
-// (k = 0 everywhere, the normal case for a pole angle), the quadrant fix-up is skipped as a whole.
-__device__ __forceinline__ void sincos2(f2 x, f2 &sn, f2 &cs, uint32_t converged_mask)
-{
-    const f2 magic = splat(kRoundMagic);
-    const f2 t = mul2(x, splat(fbits(0x3F22F983u)));
-    const f2 nb = add2(t, magic);
-    const f2 nk = sub2(magic, nb);
-    f2 r = fma2(nk, splat(fbits(0x3FC90FDBu)), x);
-    r = fma2(nk, splat(fbits(0xB33BBD2Eu)), r);
-    r = fma2(nk, splat(fbits(0xA6F72CEDu)), r);
-    const f2 r2 = mul2(r, r);
-    f2 p = fma2(splat(fbits(0x3638EF1Du)), r2, splat(fbits(0xB9500D01u)));
-    p = fma2(p, r2, splat(fbits(0x3C088889u)));
-    p = fma2(p, r2, splat(fbits(0xBE2AAAABu)));
-    const f2 S = fma2(p, mul2(r2, r), r);
-    f2 c = fma2(splat(fbits(0xB493F27Eu)), r2, splat(fbits(0x37D00D01u)));
-    c = fma2(c, r2, splat(fbits(0xBAB60B61u)));
-    c = fma2(c, r2, splat(fbits(0x3D2AAAABu)));
-    c = fma2(c, r2, splat(-0.5f));
-    const f2 C = fma2(c, r2, splat(1.0f));
-    const uint32_t qa = __float_as_uint(lo(nb)), qb = __float_as_uint(hi(nb));
-    constexpr uint32_t kMagicBits = 0x4B400000u;
-    if (__any_sync(converged_mask, ((qa ^ kMagicBits) | (qb ^ kMagicBits)) != 0u)) {
-        float sa, ca, sb, cb;
-        quadrant_fix(qa, lo(S), lo(C), sa, ca);
-        quadrant_fix(qb, hi(S), hi(C), sb, cb);
-        sn = pk(sa, sb);
-        cs = pk(ca, cb);
-    } else {
-        sn = S;
-        cs = C;
-    }
-}
-
 // Polynomial halves of sin/cos for two arguments at once (general quadrant): returns the two
 // polynomial values and the quadrant words; the callers below pick what they need.
 __device__ __forceinline__ void sincos_poly2(f2 x, f2 &S, f2 &C, uint32_t &qa, uint32_t &qb)
