@@ -78,6 +78,16 @@ int sim_set_env_offset(sim_t *s, uint64_t env_offset);
  * plain simulator).  Applies to every later sim_step / sim_rollout of the handle. */
 int sim_set_compute_factor(sim_t *s, int compute_factor);
 
+/* sim_set_action_stream -- how the uniform random policy turns Philox output into actions.
+ *   SIM_ACTIONS_WORD (default): one 32-bit word per (env, step), as described at the top of this file.
+ *   SIM_ACTIONS_BITS (CartPole only, an optional cheaper variant): one bit per (env, step): bit (t mod 128)
+ *     of the 128-bit block with counter (env, c, 2, 0), c = (low 32 bits of t div 4) div 32; bit b is bit
+ *     (b mod 32) of word (b div 32).  One Philox evaluation then serves 128 steps of an env instead of 4.
+ * The MLP policy and caller-given actions are not affected.  SIM_EINVAL for other env kinds.  (The paper
+ * names no generator; both streams are deterministic functions of (seed, env, step).) */
+enum { SIM_ACTIONS_WORD = 0, SIM_ACTIONS_BITS = 1 };
+int sim_set_action_stream(sim_t *s, int mode);
+
 /* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env. */
 int sim_reset(sim_t *s);
 

@@ -83,6 +83,13 @@ def lib() -> C.CDLL:
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_void_p]
         L.oracle_rollout_c.restype = C.c_int
+        L.oracle_rollout_x.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_int64, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_int,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_void_p]
+        L.oracle_rollout_x.restype = C.c_int
+        L.oracle_action_bit.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
+        L.oracle_action_bit.restype = C.c_int
         L.oracle_reset.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int64, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_reset.restype = C.c_int
@@ -114,6 +121,10 @@ def philox4x32_10(ctr, key):
 
 def action_word(seed, env, t):
     return int(lib().oracle_action_word(seed, env, t))
+
+
+def action_bit(seed, env, t):
+    return int(lib().oracle_action_bit(seed, env, t))
 
 
 def uniform01(w):
@@ -227,9 +238,10 @@ def sample_action(logits, w):
 class OracleSim:
     """Plain CPU stepper over a list of global env indices (default: 0..n-1)."""
 
-    def __init__(self, env_kind, n_envs=None, state_dim=4, seed=0, env_ids=None, compute_factor=1):
+    def __init__(self, env_kind, n_envs=None, state_dim=4, seed=0, env_ids=None, compute_factor=1, action_stream=0):
         self.kind, self.S, self.seed = int(env_kind), int(state_dim), int(seed)
         self.compute_factor = int(compute_factor)
+        self.action_stream = int(action_stream)
         if env_ids is None:
             env_ids = np.arange(n_envs, dtype=np.uint32)
         self.env_ids = np.ascontiguousarray(env_ids, dtype=np.uint32)
@@ -255,7 +267,7 @@ class OracleSim:
         nxt = np.zeros((T, n, S), dtype=np.float32) if "next_obs" in want else None
         pp = None if policy_params is None else _f32(policy_params)
         ga = None if actions is None else np.ascontiguousarray(actions, dtype=np.int8).reshape(T, n)
-        rc = lib().oracle_rollout_c(self.kind, S, self.seed, self.compute_factor, n, _vp(self.env_ids), _vp(self.state),
+        rc = lib().oracle_rollout_x(self.kind, S, self.seed, self.compute_factor, self.action_stream, n, _vp(self.env_ids), _vp(self.state),
                                   _vp(self.ep_len), _vp(self.reset_count), self.t, T,
                                   _vp(pp), _vp(ga), _vp(obs), _vp(act), _vp(rew), _vp(done), _vp(nxt))
         assert rc == 0, "oracle_rollout rejected its arguments"

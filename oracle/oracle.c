@@ -72,6 +72,20 @@ ORACLE_API uint32_t oracle_action_word(uint64_t seed, uint32_t env, uint64_t t)
     return blk[t & 3];
 }
 
+/* Bit-sliced action stream (an optional variant for two-action envs): the action of (env, t) is bit
+ * (t mod 128) of the 128-bit block with counter (env, c, 2, 0), c = (low 32 bits of t div 4) div 32;
+ * bit b lives in word b div 32 at position b mod 32 (least significant first). */
+ORACLE_API int oracle_action_bit(uint64_t seed, uint32_t env, uint64_t t)
+{
+    uint32_t key[2], ctr[4], blk[4];
+    seed_key(seed, key);
+    uint32_t tb = (uint32_t)(t >> 2);
+    ctr[0] = env; ctr[1] = tb >> 5; ctr[2] = 2; ctr[3] = 0;
+    oracle_philox4x32_10(ctr, key, blk);
+    uint32_t b = (uint32_t)(t & 127);
+    return (int)((blk[b >> 5] >> (b & 31)) & 1u);
+}
+
 /* u = (top 24 bits of w) * 2^-24, exact in binary32, in [0, 1 - 2^-24]. */
 ORACLE_API float oracle_uniform01(uint32_t w)
 {
@@ -403,7 +417,7 @@ ORACLE_API int oracle_sample_action(const float logits[2], uint32_t w)
  * next_obs, if not NULL, is [T,n_sel,S]: the state after step t and after auto-reset.
  * Returns 0, or -1 on bad arguments.
  * ---------------------------------------------------------------------------------- */
-ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_factor,
+ORACLE_API int oracle_rollout_x(int env_kind, int S, uint64_t seed, int compute_factor, int action_stream,
                               int64_t n_sel, const uint32_t *env_ids,
                               float *state, uint32_t *ep_len, uint32_t *reset_count,
                               uint64_t t0, int T,
@@ -415,6 +429,7 @@ ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_
     if (env_kind != ENV_SYNTH && S != 4) return -1;
     if (policy_params && env_kind != ENV_CARTPOLE) return -1;
     if (compute_factor < 1) return -1;
+    if (action_stream != 0 && (action_stream != 1 || env_kind != ENV_CARTPOLE || policy_params)) return -1;
     float cur[4096], nxt[4096], scratch[4096];
     for (int64_t e = 0; e < n_sel; ++e) {
         uint32_t env = env_ids[e];
@@ -434,7 +449,7 @@ ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_
                 oracle_mlp_logits(policy_params, cur, logits);
                 act = oracle_sample_action(logits, w);
             } else {
-                act = oracle_random_action(env_kind, w);
+                act = action_stream ? oracle_action_bit(seed, env, t) : oracle_random_action(env_kind, w);
             }
 
             /* compute factor C (paper Section 4.2): the dynamics update is iterated C times with the
@@ -474,6 +489,19 @@ ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_
         ep_len[e] = len; reset_count[e] = rc;
     }
     return 0;
+}
+
+/* Word-per-step action stream (the default). */
+ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_factor,
+                                int64_t n_sel, const uint32_t *env_ids,
+                                float *state, uint32_t *ep_len, uint32_t *reset_count,
+                                uint64_t t0, int T,
+                                const float *policy_params, const int8_t *given_actions,
+                                float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done,
+                                float *next_obs)
+{
+    return oracle_rollout_x(env_kind, S, seed, compute_factor, 0, n_sel, env_ids, state, ep_len, reset_count, t0, T,
+                            policy_params, given_actions, out_obs, out_act, out_rew, out_done, next_obs);
 }
 
 /* The plain simulator: compute factor 1. */

@@ -24,6 +24,7 @@ SIGNATURES = {
     "sim_set_stream": (C.c_int, [C.c_void_p, C.c_void_p]),
     "sim_set_env_offset": (C.c_int, [C.c_void_p, C.c_uint64]),
     "sim_set_compute_factor": (C.c_int, [C.c_void_p, C.c_int]),
+    "sim_set_action_stream": (C.c_int, [C.c_void_p, C.c_int]),
     "sim_reset": (C.c_int, [C.c_void_p]),
     "sim_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "sim_rollout": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -107,6 +108,13 @@ def sim_set_compute_factor(h, compute_factor):
     _check(lib().sim_set_compute_factor(h, compute_factor), h)
 
 
+SIM_ACTIONS_WORD, SIM_ACTIONS_BITS = 0, 1
+
+
+def sim_set_action_stream(h, mode):
+    _check(lib().sim_set_action_stream(h, mode), h)
+
+
 def sim_reset(h):
     _check(lib().sim_reset(h), h)
 
@@ -169,7 +177,7 @@ def sim_launch_count(h):
 class Sim:
     """Owning wrapper of one handle, with torch tensors for the outputs (memory plumbing only)."""
 
-    def __init__(self, env_kind, n_envs, state_dim=4, seed=0, device="cuda:0", env_offset=0, compute_factor=1):
+    def __init__(self, env_kind, n_envs, state_dim=4, seed=0, device="cuda:0", env_offset=0, compute_factor=1, action_stream=0):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -181,6 +189,8 @@ class Sim:
                 sim_reset(self.h)
             if compute_factor != 1:
                 sim_set_compute_factor(self.h, compute_factor)
+            if action_stream:
+                sim_set_action_stream(self.h, action_stream)
         self.use_stream(None)
 
     def use_stream(self, stream):

@@ -58,14 +58,25 @@ rollout_s4_kernel(const __grid_constant__ S4Args a)
     size_t row = i;                                    // element index into the [K, n] outputs
 
     const int nblk = (a.phase + a.K + 3) >> 2;         // Philox action blocks touched by this launch
+    uint4 bits_blk = make_uint4(0u, 0u, 0u, 0u);       // bit-sliced action stream: current 128-bit block
+    uint32_t bits_idx = 0u;
+    bool bits_have = false;
     for (int b = 0; b < nblk; ++b) {
         uint4 blk = make_uint4(0u, 0u, 0u, 0u);
-        if (POLICY != POLICY_GIVEN) blk = philox(env, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
+        if (POLICY != POLICY_GIVEN && !a.action_bits) blk = philox(env, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int k = 4 * b + j - a.phase;         // step index inside the launch (warp-uniform)
             if (k < 0 || k >= a.K) continue;
-            const uint32_t w = j == 0 ? blk.x : j == 1 ? blk.y : j == 2 ? blk.z : blk.w;
+            uint32_t w = j == 0 ? blk.x : j == 1 ? blk.y : j == 2 ? blk.z : blk.w;
+            if (POLICY == POLICY_RANDOM && ENV == ENV_CARTPOLE && a.action_bits) {
+                // bit-sliced stream: bit (t mod 128) of the block with counter (env, (t >> 2) >> 5, 2, 0)
+                const uint32_t tb = a.tb0 + (uint32_t)b;
+                if (!bits_have || (tb >> 5) != bits_idx) { bits_blk = philox(env, tb >> 5, 2u, 0u, a.rk); bits_idx = tb >> 5; bits_have = true; }
+                const uint32_t bi = ((tb & 31u) << 2) | (uint32_t)j;
+                const uint32_t word = (bi >> 5) == 0 ? bits_blk.x : (bi >> 5) == 1 ? bits_blk.y : (bi >> 5) == 2 ? bits_blk.z : bits_blk.w;
+                w = (word >> (bi & 31u)) << 31;
+            }
 
             if (a.out_obs) __stcs(&a.out_obs[row], s);
 

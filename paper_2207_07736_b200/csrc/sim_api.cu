@@ -19,6 +19,7 @@ struct sim {
     uint64_t env_offset;
     uint64_t t;
     int compute_factor;
+    int action_stream;
     int device;
     cudaStream_t stream;
     float *state;
@@ -151,6 +152,14 @@ SIM_API int sim_set_compute_factor(sim_t *s, int compute_factor)
     return SIM_OK;
 }
 
+SIM_API int sim_set_action_stream(sim_t *s, int mode)
+{
+    if (!s || (mode != SIM_ACTIONS_WORD && mode != SIM_ACTIONS_BITS)) return SIM_EINVAL;
+    if (mode == SIM_ACTIONS_BITS && s->env_kind != SIM_CARTPOLE) return SIM_EINVAL;
+    s->action_stream = mode;
+    return SIM_OK;
+}
+
 SIM_API int sim_reset(sim_t *s)
 {
     if (!s) return SIM_EINVAL;
@@ -179,6 +188,7 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
         a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = s->compute_factor;
         a.out_obs = reinterpret_cast<float4 *>(obs); a.out_act = act; a.out_rew = rew; a.out_done = done;
         a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.rk = s->rk;
+        a.action_bits = (s->action_stream == SIM_ACTIONS_BITS && policy == POLICY_RANDOM) ? 1 : 0;
         if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM && s->compute_factor == 1)
             CU(s, launch_cartpole_random(a, s->stream));
         else if (s->env_kind == SIM_ACROBOT && policy == POLICY_RANDOM && K > 4)      // short launches: the scalar kernel has the shorter step latency

@@ -20,6 +20,7 @@ struct S4Args {
     int phase;                // t0 & 3
     int K;                    // steps in this launch
     int C;                    // compute factor: dynamics iterations per recorded step (>= 1)
+    int action_bits;          // 1: bit-sliced action stream (CartPole, random policy)
     float4 *out_obs;          // [K, n] or nullptr
     int8_t *out_act;          // [K, n] or nullptr
     float *out_rew;           // [K, n] or nullptr

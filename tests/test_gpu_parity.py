@@ -335,6 +335,32 @@ def test_random_shapes_against_the_oracle():
         compare_rollout(out, sim, ref, orc, what="case %d kind %d S %d n %d T %d K %d C %d" % (case, kind, S, n, T, K, C))
 
 
+@pytest.mark.parametrize("K", [1, 5, 8, 13, 64, 300])
+def test_bit_sliced_action_stream(K):
+    """The optional one-bit-per-step action stream: windows aligned to bytes of action bits, launches starting
+    at every offset inside a 128-step block, block boundaries inside a launch, the generic kernel (C > 1)."""
+    torch = torch_cuda()
+    for t0, C in ((0, 1), (121, 1), ((1 << 34) + 3, 1), (6, 2)):
+        sim = binding.Sim(oracle.CARTPOLE, 333, 4, 19, compute_factor=C, action_stream=binding.SIM_ACTIONS_BITS)
+        orc = oracle.OracleSim(oracle.CARTPOLE, 333, 4, 19, compute_factor=C, action_stream=1)
+        ep, rc, _ = sim.counters()
+        sim.set_counters(ep, rc, t0)
+        orc.t = t0
+        out = sim.rollout(300, K)
+        torch.cuda.synchronize()
+        ref = orc.rollout(300)
+        compare_rollout(out, sim, ref, orc, what="bits K=%d t0=%d C=%d" % (K, t0, C))
+    L = binding.lib()
+    acro = binding.Sim(oracle.ACROBOT, 8)
+    assert L.sim_set_action_stream(acro.h, binding.SIM_ACTIONS_BITS) == binding.SIM_EINVAL
+    assert L.sim_set_action_stream(acro.h, 7) == binding.SIM_EINVAL and L.sim_set_action_stream(None, 0) == binding.SIM_EINVAL
+    # the MLP policy is unaffected by the stream mode
+    p = torch.from_numpy(inputs.mlp_params(1)).cuda()
+    a = binding.Sim(oracle.CARTPOLE, 100, 4, 2, action_stream=binding.SIM_ACTIONS_BITS).rollout(20, 20, p)
+    b = binding.Sim(oracle.CARTPOLE, 100, 4, 2).rollout(20, 20, p)
+    assert torch.equal(a["act"], b["act"]) and torch.equal(a["obs"], b["obs"])
+
+
 def test_argument_errors_with_live_handle():
     torch = torch_cuda()
     sim = binding.Sim(oracle.ACROBOT, 16)

@@ -90,3 +90,20 @@ def test_action_stream_statistics():
     tern = ((w * np.uint64(3)) >> np.uint64(32)).astype(int)
     counts = np.bincount(tern, minlength=3)
     assert np.all(np.abs(counts / n - 1 / 3) < 4 * np.sqrt(2 / 9 / n))
+
+
+def test_bit_sliced_action_stream():
+    seed = 77
+    for env, t in [(0, 0), (3, 1), (3, 31), (3, 32), (3, 127), (3, 128), (9, 1000), (5, (1 << 34) + 77)]:
+        tb = (t >> 2) & 0xFFFFFFFF
+        blk = oracle.philox4x32_10([env, tb >> 5, 2, 0], [seed, 0])
+        b = t & 127
+        assert oracle.action_bit(seed, env, t) == (int(blk[b >> 5]) >> (b & 31)) & 1
+    bits = np.array([oracle.action_bit(1, e, t) for e in range(16) for t in range(1024)])
+    assert abs(bits.mean() - 0.5) < 4 * 0.5 / np.sqrt(bits.size)
+    # a rollout in this mode takes exactly these actions, and differs from the word stream
+    a = oracle.OracleSim(oracle.CARTPOLE, 8, seed=1, action_stream=1).rollout(300)
+    want = np.array([[oracle.action_bit(1, e, t) for e in range(8)] for t in range(300)], dtype=np.int8)
+    assert np.array_equal(a["act"], want)
+    b = oracle.OracleSim(oracle.CARTPOLE, 8, seed=1).rollout(300)
+    assert not np.array_equal(a["act"], b["act"])
