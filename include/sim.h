@@ -149,6 +149,14 @@ int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_pa
  * bit.  (The paper's simulators expose raw state only; this is a convenience on top of the path.) */
 int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, float *d_obs6);
 
+/* sim_episode_returns -- running return of every episode of a trajectory, for consumers that label the
+ * collected samples with returns (the paper: "reward is used to form labels for the collected data",
+ * Section 2.1).  d_rew [T,n] fp32 and d_done [T,n] u8 as written by sim_rollout; d_ret [T,n] fp32 receives
+ * ret[t,e] = rew[t,e] + (done[t-1,e] ? 0 : ret[t-1,e]), added in time order in fp32.  d_carry [n] fp32
+ * (nullable) carries the return accumulated so far across calls: read before row 0, written after the last
+ * row (0 where the episode just ended).  All device pointers. */
+int sim_episode_returns(sim_t *s, const float *d_rew, const uint8_t *d_done, int T, int64_t n, float *d_carry, float *d_ret);
+
 /* sim_selfcheck_division -- numerical self-check of the divisions inside the fused kernels (the paper
  * has no counterpart; it exists so a test can prove the kernels' arithmetic on the device they run
  * on).  The fused CartPole and Acrobot kernels divide by well-conditioned denominators with a refined

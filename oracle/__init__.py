@@ -90,6 +90,8 @@ def lib() -> C.CDLL:
         L.oracle_rollout_x.restype = C.c_int
         L.oracle_action_bit.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
         L.oracle_action_bit.restype = C.c_int
+        L.oracle_episode_returns.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_void_p]
+        L.oracle_episode_returns.restype = None
         L.oracle_reset.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int64, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_reset.restype = C.c_int
@@ -232,6 +234,16 @@ def mlp_logits(params, obs):
 def sample_action(logits, w):
     logits = _f32(logits)
     return int(lib().oracle_sample_action(_fp(logits), int(w)))
+
+
+def episode_returns(rew, done, carry=None):
+    rew = np.ascontiguousarray(rew, dtype=np.float32)
+    done = np.ascontiguousarray(done, dtype=np.uint8)
+    T, n = rew.shape
+    carry = np.zeros(n, dtype=np.float32) if carry is None else np.ascontiguousarray(carry, dtype=np.float32).copy()
+    ret = np.zeros((T, n), dtype=np.float32)
+    lib().oracle_episode_returns(_vp(rew), _vp(done), T, n, _vp(carry), _vp(ret))
+    return ret, carry
 
 
 # ---------------------------------------------------------------- whole pipeline

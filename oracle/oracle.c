@@ -517,6 +517,21 @@ ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
                             policy_params, given_actions, out_obs, out_act, out_rew, out_done, next_obs);
 }
 
+/* Running return of every episode in a trajectory: ret[t,e] = rew[t,e] + (done[t-1,e] ? 0 : ret[t-1,e]),
+ * with `carry` [n] (in: return accumulated before row 0; out: after the last row, 0 where it ended). */
+ORACLE_API void oracle_episode_returns(const float *rew, const uint8_t *done, int T, int64_t n, float *carry, float *ret)
+{
+    for (int64_t e = 0; e < n; ++e) {
+        float acc = carry[e];
+        for (int t = 0; t < T; ++t) {
+            acc = acc + rew[(size_t)t * (size_t)n + (size_t)e];
+            ret[(size_t)t * (size_t)n + (size_t)e] = acc;
+            if (done[(size_t)t * (size_t)n + (size_t)e]) acc = 0.0f;
+        }
+        carry[e] = acc;
+    }
+}
+
 /* Initial condition (draw #0, zeroed counters) for a list of env indices. */
 ORACLE_API int oracle_reset(int env_kind, int S, uint64_t seed, int64_t n_sel, const uint32_t *env_ids,
                             float *state, uint32_t *ep_len, uint32_t *reset_count)

@@ -35,6 +35,7 @@ SIGNATURES = {
     "sim_set_counters": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]),
     "sim_policy_logits": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]),
     "sim_acrobot_observation": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
+    "sim_episode_returns": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_void_p, C.c_void_p]),
     "sim_selfcheck_division": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_uint64)]),
     "sim_rollout_noalloc": (C.c_int, [C.c_int, C.c_int64, C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -155,6 +156,10 @@ def sim_policy_logits(h, d_obs, M, d_params, d_logits):
 
 def sim_acrobot_observation(h, d_state, M, d_obs6):
     _check(lib().sim_acrobot_observation(h, _ptr(d_state), M, _ptr(d_obs6)), h)
+
+
+def sim_episode_returns(h, d_rew, d_done, T, n, d_carry, d_ret):
+    _check(lib().sim_episode_returns(h, _ptr(d_rew), _ptr(d_done), T, n, _ptr(d_carry), _ptr(d_ret)), h)
 
 
 def sim_selfcheck_division(h, nums_per_den):

@@ -160,6 +160,32 @@ cudaError_t launch_acrobot_observation(const float *state, int64_t M, float *obs
     return cudaGetLastError();
 }
 
+// Running episode return over a trajectory: one thread per env walks the T rows (each row access of a
+// warp is contiguous), adding in time order, restarting after a done.
+__global__ void __launch_bounds__(256)
+episode_returns_kernel(const float *__restrict__ rew, const uint8_t *__restrict__ done, int T, int64_t n, float *carry, float *__restrict__ ret)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n) return;
+    float acc = carry ? carry[e] : 0.0f;
+    for (int t = 0; t < T; ++t) {
+        const size_t at = (size_t)t * (size_t)n + (size_t)e;
+        acc = __fadd_rn(acc, rew[at]);
+        ret[at] = acc;
+        if (done[at]) acc = 0.0f;
+    }
+    if (carry) carry[e] = acc;
+}
+
+cudaError_t launch_episode_returns(const float *rew, const uint8_t *done, int T, int64_t n, float *carry, float *ret, cudaStream_t st)
+{
+    if (n <= 0 || T <= 0) return cudaSuccess;
+    const int64_t blocks = (n + 255) / 256;
+    if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
+    episode_returns_kernel<<<(unsigned)blocks, 256, 0, st>>>(rew, done, T, n, carry, ret);
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------------------------
 // Launchers
 // ---------------------------------------------------------------------------------------------

@@ -368,3 +368,11 @@ SIM_API int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, f
     if (M > 0) s->launches += 1;
     return SIM_OK;
 }
+
+SIM_API int sim_episode_returns(sim_t *s, const float *d_rew, const uint8_t *d_done, int T, int64_t n, float *d_carry, float *d_ret)
+{
+    if (!s || !d_rew || !d_done || !d_ret || T < 0 || n < 0) return SIM_EINVAL;
+    CU(s, launch_episode_returns(d_rew, d_done, T, n, d_carry, d_ret, s->stream));
+    if (T > 0 && n > 0) s->launches += 1;
+    return SIM_OK;
+}

@@ -86,6 +86,7 @@ cudaError_t launch_cartpole_mlp(const S4Args &a, cudaStream_t st);      // CartP
 cudaError_t launch_division_selfcheck(int nums_per_den, unsigned long long *d_bad, cudaStream_t st);
 cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st);
 cudaError_t launch_acrobot_observation(const float *state, int64_t M, float *obs6, cudaStream_t st);
+cudaError_t launch_episode_returns(const float *rew, const uint8_t *done, int T, int64_t n, float *carry, float *ret, cudaStream_t st);
 cudaError_t launch_policy_logits(const float *obs, int64_t M, const float *params, float *logits, cudaStream_t st);
 
 }  // namespace simk

@@ -361,6 +361,20 @@ def test_bit_sliced_action_stream(K):
     assert torch.equal(a["act"], b["act"]) and torch.equal(a["obs"], b["obs"])
 
 
+def test_episode_returns_entry_point():
+    torch = torch_cuda()
+    for kind in (oracle.CARTPOLE, oracle.ACROBOT):
+        sim = binding.Sim(kind, 777, 4, 3)
+        out = sim.rollout(530, 530)
+        ret = torch.empty_like(out["rew"])
+        carry = torch.zeros(777, dtype=torch.float32, device="cuda")
+        binding.sim_episode_returns(sim.h, out["rew"][:200], out["done"][:200], 200, 777, carry, ret[:200])
+        binding.sim_episode_returns(sim.h, out["rew"][200:], out["done"][200:], 330, 777, carry, ret[200:])
+        want, wc = oracle.episode_returns(to_np(out["rew"]), to_np(out["done"]))
+        assert_same_bits(to_np(ret), want, "returns")
+        assert_same_bits(to_np(carry), wc, "carry")
+
+
 def test_argument_errors_with_live_handle():
     torch = torch_cuda()
     sim = binding.Sim(oracle.ACROBOT, 16)

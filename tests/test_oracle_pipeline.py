@@ -109,3 +109,27 @@ def test_compute_factor_is_iterated_dynamics_with_the_action_held():
     first = np.array([np.flatnonzero(out["done"][:, e])[0] for e in range(256)])
     assert 1 <= first.min() and first.mean() < 8
     assert np.array_equal(fat.reset_count, out["done"].sum(0).astype(np.uint32))
+
+
+def test_episode_returns():
+    sim = oracle.OracleSim(oracle.CARTPOLE, 40, seed=3)
+    out = sim.rollout(120)
+    ret, carry = oracle.episode_returns(out["rew"], out["done"])
+    done = out["done"].astype(bool)
+    for e in range(40):
+        steps = 0
+        for t in range(120):
+            steps += 1
+            assert ret[t, e] == steps              # CartPole pays 1 per step: the return is the step count of the episode
+            if done[t, e]:
+                steps = 0
+        assert carry[e] == steps == sim.ep_len[e]
+    # split in two calls with the carry
+    r1, c1 = oracle.episode_returns(out["rew"][:50], out["done"][:50])
+    r2, c2 = oracle.episode_returns(out["rew"][50:], out["done"][50:], c1)
+    assert np.array_equal(np.concatenate([r1, r2]), ret) and np.array_equal(c2, carry)
+    # Acrobot: -1 per step, 0 on the goal step
+    ac = oracle.OracleSim(oracle.ACROBOT, 16, seed=1)
+    o = ac.rollout(600)
+    r, _ = oracle.episode_returns(o["rew"], o["done"])
+    assert r[498, 0] == -499.0 and r.min() >= -500.0
