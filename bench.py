@@ -239,7 +239,8 @@ def run_gpu(args, w):
     env_offset, n = shard.env_range(rank, world, w.n_envs)
     K = args.k_fused or max(w.k_sweep)
     sim = binding.Sim(w.env_kind, n, w.state_dim, w.seed, device=dev, env_offset=env_offset, compute_factor=args.compute_factor,
-                      action_stream=1 if args.action_bits else 0)
+                      action_stream=1 if args.action_bits else 0,
+                      policy_mode=binding.SIM_POLICY_TENSOR if args.policy_mode == "tensor" else binding.SIM_POLICY_EXACT)
     d_params = None if w.mlp_seed is None else torch.from_numpy(inputs.mlp_params(w.mlp_seed)).to(dev)
     out = sim.alloc_outputs(w.T) if w.trajectory else {}
     traj_bytes = sum(t.numel() * t.element_size() for t in out.values() if t is not None)
@@ -381,7 +382,7 @@ def run_gpu(args, w):
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "env": ["cartpole", "acrobot", "synthetic"][w.env_kind], "n_envs_per_gpu": n, "T": w.T,
-                   "state_dim": w.state_dim, "k_fused": K, "compute_factor": args.compute_factor, "action_stream": "bits" if args.action_bits else "word", "policy": "mlp_4_64_64_2" if w.mlp_seed is not None else "uniform_random",
+                   "state_dim": w.state_dim, "k_fused": K, "compute_factor": args.compute_factor, "action_stream": "bits" if args.action_bits else "word", "policy": "mlp_4_64_64_2" if w.mlp_seed is not None else "uniform_random", "policy_mode": args.policy_mode,
                    "trajectory_bytes_per_step": traj_bytes,
                    "l2": "each step writes %.2f GB of trajectory (> 126 MB L2); no flush between steps" % (traj_bytes / 1e9) if traj_bytes > 2e8
                    else "state (%.2f GB) streamed from HBM every launch" % (n * w.state_dim * 4 / 1e9),
@@ -435,6 +436,8 @@ def main():
     ap.add_argument("--n-envs", type=int, default=0, help="override the workload's env count (profiling on a reduced case)")
     ap.add_argument("--T", type=int, default=0, help="override the workload's step count (profiling on a reduced case)")
     ap.add_argument("--compute-factor", type=int, default=1, help="dynamics iterations per recorded step (the paper's knob C)")
+    ap.add_argument("--policy-mode", choices=("exact", "tensor"), default="exact",
+                    help="MLP policy evaluation: exact fp32 (default) or tolerance mode with the hidden layer on the tensor cores")
     ap.add_argument("--action-bits", action="store_true", help="optional bit-sliced action stream (CartPole random policy; not the default workload)")
     ap.add_argument("--grid", action="store_true", help="fusion speedup over the S x C x K simulator-complexity grid (synthetic simulator)")
     ap.add_argument("--no-sweep", action="store_true")

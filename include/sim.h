@@ -88,6 +88,33 @@ int sim_set_compute_factor(sim_t *s, int compute_factor);
 enum { SIM_ACTIONS_WORD = 0, SIM_ACTIONS_BITS = 1 };
 int sim_set_action_stream(sim_t *s, int mode);
 
+/* sim_set_policy_mode -- how the MLP policy is evaluated inside sim_rollout / sim_rollout_host /
+ * sim_policy_logits (CartPole only; SIM_EINVAL for other env kinds or an unknown mode).
+ *   SIM_POLICY_EXACT (default): the fp32 definition at the top of this file; actions are bit-reproducible.
+ *   SIM_POLICY_TENSOR: tolerance mode for throughput (the fusion of simulation and inference that
+ *     Section 7 of the paper leaves as future work, with the hidden layer on the tensor cores):
+ *       h1 = tanh~(W1 obs + b1)            layer-1 sums as in exact mode; tanh~ = the GPU's approximate
+ *                                          tanh instruction (relative error about 2^-11)
+ *       z2 = b2 + sum_k tf32(W2[j][k]) * tf32(h1[k])   operands rounded to TF32 (10-bit mantissa,
+ *                                          round to nearest, ties away), products exact, fp32 accumulation
+ *                                          in the order the tensor core chooses
+ *       h2 = tanh~(z2);  logits = b3 + W3 h2 in fp32, ascending j.
+ *     Sampling, physics, reset and outputs are unchanged, so a trajectory stays an exact CartPole
+ *     trajectory under the actions it records; only the action probabilities differ from exact mode,
+ *     by the logit error (bounded by sum_j |W3[i][j]| (eps + sum_k |W2[j][k]| (eps + 2^-10)) with
+ *     eps = 2^-10.9, far less for typical weights).  Not bit-reproducible across GPU generations.
+ * The first call that selects tensor mode allocates a 4-byte device status word (see
+ * sim_get_device_status). */
+enum { SIM_POLICY_EXACT = 0, SIM_POLICY_TENSOR = 1 };
+int sim_set_policy_mode(sim_t *s, int mode);
+
+/* sim_get_device_status -- flags raised by kernels of this handle since it was created; synchronises the
+ * handle's stream.  h_flags is a HOST pointer.  Bit 0 (SIM_STATUS_TENSOR_WAIT): a tensor-mode kernel gave
+ * up waiting for the tensor core (every such wait is bounded, about a second); the rollout that hit it
+ * left states and outputs of the affected envs unspecified.  0 when tensor mode was never selected. */
+enum { SIM_STATUS_TENSOR_WAIT = 1 };
+int sim_get_device_status(sim_t *s, uint32_t *h_flags);
+
 /* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env. */
 int sim_reset(sim_t *s);
 
@@ -139,7 +166,7 @@ int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t *d_reset
 
 /* sim_policy_logits -- logits of the MLP for M observations (no sampling, no stepping).
  *   d_obs [M,4] fp32, d_params SIM_POLICY_PARAM_COUNT fp32, d_logits [M,2] fp32.  s may be
- *   any live handle (it provides the stream). */
+ *   any live handle (it provides the stream and the policy mode). */
 int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits);
 
 /* sim_acrobot_observation -- the six-value observation an RL consumer of Acrobot usually wants,

@@ -25,6 +25,8 @@ SIGNATURES = {
     "sim_set_env_offset": (C.c_int, [C.c_void_p, C.c_uint64]),
     "sim_set_compute_factor": (C.c_int, [C.c_void_p, C.c_int]),
     "sim_set_action_stream": (C.c_int, [C.c_void_p, C.c_int]),
+    "sim_set_policy_mode": (C.c_int, [C.c_void_p, C.c_int]),
+    "sim_get_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint32)]),
     "sim_reset": (C.c_int, [C.c_void_p]),
     "sim_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "sim_rollout": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -116,6 +118,20 @@ def sim_set_action_stream(h, mode):
     _check(lib().sim_set_action_stream(h, mode), h)
 
 
+SIM_POLICY_EXACT, SIM_POLICY_TENSOR = 0, 1
+SIM_STATUS_TENSOR_WAIT = 1
+
+
+def sim_set_policy_mode(h, mode):
+    _check(lib().sim_set_policy_mode(h, mode), h)
+
+
+def sim_get_device_status(h) -> int:
+    flags = C.c_uint32(0)
+    _check(lib().sim_get_device_status(h, C.byref(flags)), h)
+    return flags.value
+
+
 def sim_reset(h):
     _check(lib().sim_reset(h), h)
 
@@ -182,7 +198,7 @@ def sim_launch_count(h):
 class Sim:
     """Owning wrapper of one handle, with torch tensors for the outputs (memory plumbing only)."""
 
-    def __init__(self, env_kind, n_envs, state_dim=4, seed=0, device="cuda:0", env_offset=0, compute_factor=1, action_stream=0):
+    def __init__(self, env_kind, n_envs, state_dim=4, seed=0, device="cuda:0", env_offset=0, compute_factor=1, action_stream=0, policy_mode=0):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -196,6 +212,8 @@ class Sim:
                 sim_set_compute_factor(self.h, compute_factor)
             if action_stream:
                 sim_set_action_stream(self.h, action_stream)
+            if policy_mode:
+                sim_set_policy_mode(self.h, policy_mode)
         self.use_stream(None)
 
     def use_stream(self, stream):
@@ -273,6 +291,10 @@ class Sim:
         with self.torch.cuda.device(self.device):
             sim_policy_logits(self.h, obs, obs.shape[0], params, out)
         return out
+
+    def device_status(self):
+        with self.torch.cuda.device(self.device):
+            return sim_get_device_status(self.h)
 
     @property
     def launches(self):

@@ -110,17 +110,6 @@ __device__ __forceinline__ void mlp_logits2(const float4 oa, const float4 ob, co
     }
 }
 
-// Inverse-CDF sample over the two unnormalised softmax weights: action 0 iff u*(e0+e1) < e0.
-__device__ __forceinline__ int sample_pair(f2 l, uint32_t w)
-{
-    const float m = fmaxf(lo(l), hi(l));
-    const float y0 = fminf(fmaxf(__fsub_rn(lo(l), m), -87.0f), 88.0f);
-    const float y1 = fminf(fmaxf(__fsub_rn(hi(l), m), -87.0f), 88.0f);
-    const f2 e = exp2_core(pk(y0, y1));
-    const float thr = __fmul_rn(uniform01(w), __fadd_rn(lo(e), hi(e)));
-    return (thr < lo(e)) ? 0 : 1;
-}
-
 #ifndef MLP_THREADS
 #define MLP_THREADS 128
 #endif

@@ -20,6 +20,8 @@ struct sim {
     uint64_t t;
     int compute_factor;
     int action_stream;
+    int policy_mode;
+    uint32_t *d_status;       // device status word, allocated when tensor mode is first selected
     int device;
     cudaStream_t stream;
     float *state;
@@ -88,6 +90,7 @@ static void free_handle(sim *s)
         if (s->ev_copied[i]) cudaEventDestroy(s->ev_copied[i]);
     }
     if (s->d_params) cudaFree(s->d_params);
+    if (s->d_status) cudaFree(s->d_status);
     if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
     delete s;
 }
@@ -160,6 +163,28 @@ SIM_API int sim_set_action_stream(sim_t *s, int mode)
     return SIM_OK;
 }
 
+SIM_API int sim_set_policy_mode(sim_t *s, int mode)
+{
+    if (!s || (mode != SIM_POLICY_EXACT && mode != SIM_POLICY_TENSOR)) return SIM_EINVAL;
+    if (mode == SIM_POLICY_TENSOR && s->env_kind != SIM_CARTPOLE) return SIM_EINVAL;
+    if (mode == SIM_POLICY_TENSOR && !s->d_status) {
+        CU(s, cudaMalloc(&s->d_status, sizeof(uint32_t)));
+        CU(s, cudaMemsetAsync(s->d_status, 0, sizeof(uint32_t), s->stream));
+    }
+    s->policy_mode = mode;
+    return SIM_OK;
+}
+
+SIM_API int sim_get_device_status(sim_t *s, uint32_t *h_flags)
+{
+    if (!s || !h_flags) return SIM_EINVAL;
+    *h_flags = 0u;
+    if (!s->d_status) return SIM_OK;
+    CU(s, cudaMemcpyAsync(h_flags, s->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s->stream));
+    CU(s, cudaStreamSynchronize(s->stream));
+    return SIM_OK;
+}
+
 SIM_API int sim_reset(sim_t *s)
 {
     if (!s) return SIM_EINVAL;
@@ -187,12 +212,14 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
         a.state = reinterpret_cast<float4 *>(s->state); a.ep_len = s->ep_len; a.reset_count = s->reset_count;
         a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = s->compute_factor;
         a.out_obs = reinterpret_cast<float4 *>(obs); a.out_act = act; a.out_rew = rew; a.out_done = done;
-        a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.rk = s->rk;
+        a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.status = s->d_status; a.rk = s->rk;
         a.action_bits = (s->action_stream == SIM_ACTIONS_BITS && policy == POLICY_RANDOM) ? 1 : 0;
         if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM && s->compute_factor == 1)
             CU(s, launch_cartpole_random(a, s->stream));
         else if (s->env_kind == SIM_ACROBOT && policy == POLICY_RANDOM && K > 4)      // short launches: the scalar kernel has the shorter step latency
             CU(s, launch_acrobot_random(a, s->stream));
+        else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP && s->policy_mode == SIM_POLICY_TENSOR)
+            CU(s, launch_cartpole_mlp_tc(a, s->stream));
         else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP)
             CU(s, launch_cartpole_mlp(a, s->stream));
         else
@@ -339,7 +366,10 @@ SIM_API int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t 
 SIM_API int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits)
 {
     if (!s || !d_obs || !d_params || !d_logits || M < 0) return SIM_EINVAL;
-    CU(s, launch_policy_logits(d_obs, M, d_params, d_logits, s->stream));
+    if (s->policy_mode == SIM_POLICY_TENSOR)
+        CU(s, launch_policy_logits_tc(d_obs, M, d_params, d_logits, s->d_status, s->stream));
+    else
+        CU(s, launch_policy_logits(d_obs, M, d_params, d_logits, s->stream));
     if (M > 0) s->launches += 1;
     return SIM_OK;
 }

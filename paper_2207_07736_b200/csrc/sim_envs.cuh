@@ -22,6 +22,18 @@ __device__ __forceinline__ float4 draw_state4(uint32_t env, uint32_t r, uint32_t
     return make_float4(uniform_range(b.x, w, lo), uniform_range(b.y, w, lo), uniform_range(b.z, w, lo), uniform_range(b.w, w, lo));
 }
 
+// Categorical sample of the two-action policy from its logits l = (logit0, logit1) and one Philox word:
+// inverse CDF over the two unnormalised softmax weights: action 0 iff u*(e0+e1) < e0.
+__device__ __forceinline__ int sample_pair(f2 l, uint32_t w)
+{
+    const float m = fmaxf(lo(l), hi(l));
+    const float y0 = fminf(fmaxf(__fsub_rn(lo(l), m), -87.0f), 88.0f);
+    const float y1 = fminf(fmaxf(__fsub_rn(hi(l), m), -87.0f), 88.0f);
+    const f2 e = exp2_core(pk(y0, y1));
+    const float thr = __fmul_rn(uniform01(w), __fadd_rn(lo(e), hi(e)));
+    return (thr < lo(e)) ? 0 : 1;
+}
+
 // CartPole: explicit Euler with tau = 0.02; state (x, x_dot, theta, theta_dot).
 // Returns done; reward is 1 on every step.
 __device__ __forceinline__ bool cartpole_step(float4 &s, bool push_right)

@@ -28,6 +28,7 @@ struct S4Args {
     const int8_t *actions;    // [n], POLICY_GIVEN only
     float4 *next_obs;         // [n] post-step state, POLICY_GIVEN only (nullable)
     const float *params;      // MLP parameters, POLICY_MLP only
+    uint32_t *status;         // device status word (tensor-mode policy: bit 0 = a bounded wait ran out), nullable
     RoundKeys rk;
 };
 
@@ -83,6 +84,8 @@ cudaError_t launch_s4(int env_kind, int policy, const S4Args &a, cudaStream_t st
 cudaError_t launch_cartpole_random(const S4Args &a, cudaStream_t st);   // CartPole, uniform random policy, packed two-env kernel
 cudaError_t launch_acrobot_random(const S4Args &a, cudaStream_t st);    // Acrobot, uniform random torque, packed two-env kernel
 cudaError_t launch_cartpole_mlp(const S4Args &a, cudaStream_t st);      // CartPole, MLP policy, packed two-env kernel
+cudaError_t launch_cartpole_mlp_tc(const S4Args &a, cudaStream_t st);   // CartPole, MLP policy in tensor mode (tcgen05 hidden layer)
+cudaError_t launch_policy_logits_tc(const float *obs, int64_t M, const float *params, float *logits, uint32_t *status, cudaStream_t st);
 cudaError_t launch_division_selfcheck(int nums_per_den, unsigned long long *d_bad, cudaStream_t st);
 cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st);
 cudaError_t launch_acrobot_observation(const float *state, int64_t M, float *obs6, cudaStream_t st);

@@ -105,7 +105,7 @@ int sim_rollout_noalloc(int env_kind, int64_t n_envs, int state_dim, uint64_t se
             a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k; a.C = 1;
             a.out_obs = out_obs ? reinterpret_cast<float4 *>(out_obs) + r0 : nullptr; a.out_act = out_act ? out_act + r0 : nullptr;
             a.out_rew = out_rew ? out_rew + r0 : nullptr; a.out_done = out_done ? out_done + r0 : nullptr;
-            a.actions = nullptr; a.next_obs = nullptr; a.params = d_policy_params; a.rk = rk; a.action_bits = 0;
+            a.actions = nullptr; a.next_obs = nullptr; a.params = d_policy_params; a.status = nullptr; a.rk = rk; a.action_bits = 0;
             if (env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM) e = launch_cartpole_random(a, st);
             else if (env_kind == SIM_CARTPOLE) e = launch_cartpole_mlp(a, st);
             else e = launch_s4(env_kind, policy, a, st);
