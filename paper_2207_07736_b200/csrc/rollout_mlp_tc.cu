@@ -1,64 +1,70 @@
 // Fused CartPole rollout with the MLP policy in TENSOR mode (tolerance mode, not bit-exact): all three
-// layers of the 4-64-64-2 network run on the 5th-generation tensor cores (tcgen05, accumulators in
-// TMEM), tanh is the packed half-precision hardware approximation.  The paper names fusing simulation
-// and inference as future work (Section 7); this is that fusion.
+// layers of the 4-64-64-2 network run on the 5th-generation tensor cores (tcgen05, FP16 operands, fp32
+// accumulators in TMEM), tanh is the packed half-precision hardware approximation.  The paper names
+// fusing simulation and inference as future work (Section 7); this is that fusion.
 //
-// One CTA = 128 threads = 128 envs = the 128 rows (TMEM lanes) of every accumulator.  Per step, three
-// contractions, each issued by one thread and awaited by all through an mbarrier:
-//   1. z1[128x64] = A1[128x16] B1^T    TF32; A1 row = (o_hi, o_lo, o_hi, 1, 1, 0, 0), B1 row j =
-//      (w_hi, w_hi, w_lo, b_hi, b_lo, 0, 0): observation and weights split into two TF32 parts, so the
-//      layer-1 sums carry about 21 bits, bias included;
-//   2. z2[128x64] = A2[128x80] B2^T    FP16 operands, fp32 accumulation; A2 row = (h1[0..63], 1, 1, 0...)
-//      with h1 = tanh.approx.f16x2(z1), B2 row j = (f16(W2[j][.]), b2 hi, b2 lo, 0...);
-//   3. l[128x16]  = A2'[128x80] B3^T   A2' = the same tile refilled with h2 = tanh.approx.f16x2(z2);
+// One CTA = 256 threads = two groups of 128 threads; a group owns one tile of 128 envs (thread = env =
+// row of the operand tile = TMEM lane of the accumulator) and synchronises on its own named barrier and
+// its own mbarrier, so the two groups drift apart and one converts while the other's contraction runs.
+// The weight tiles are shared by the groups.  Per step and tile, three contractions, each issued by the
+// group's first thread and awaited by the group through the mbarrier:
+//   1. z1[128x64] = A1[128x16] B1^T   A1 row = (o_hi[4], o_lo[4], o_hi[4], 1, 1, 0, 0), B1 row j =
+//      (w_hi[4], w_hi[4], w_lo[4], b_hi, b_lo, 0, 0): observation, weights and bias split into two FP16
+//      parts each, so the layer-1 sums carry about 21 bits;
+//   2. z2[128x64] = A2[128x80] B2^T   A2 row = (h1[0..63], 1, 1, 0...), h1 = tanh.approx.f16x2(z1);
+//      B2 row j = (f16(W2[j][.]), b2 hi, b2 lo, 0...);
+//   3. l[128x16]  = A2'[128x80] B3^T  A2' = the same tile refilled with h2 = tanh.approx.f16x2(z2);
 //      B3 rows 0..3 = W3[0] hi, W3[0] lo, W3[1] hi, W3[1] lo (b3 in the bias columns of the hi rows):
 //      logit i = l[2i] + l[2i+1].
-// Each thread converts its own accumulator row (tcgen05.ld, 32 lanes x 32 bit) to the next operand row,
+// Each thread converts its own accumulator row (tcgen05.ld, 32 lanes x 32 bit) into the next operand row,
 // then samples, steps the physics, resets and stores exactly like the exact kernel.
 // Operand layout in shared memory (all operands K-major, no swizzle): 8-row x 16-byte core matrices;
 // the core matrices of one 8-row group along K are contiguous (128 bytes apart = leading byte offset),
-// 8-row groups follow each other (stride byte offset = 128 bytes x 16-byte chunks per row).
-// Every wait is bounded: when a barrier does not complete in time the CTA records bit 0 in the status
-// word, skips the remaining steps, frees its TMEM columns and returns.
+// 8-row groups follow each other (stride byte offset = 128 bytes x 16-byte chunks per row).  A1 lives in
+// the first 4 KB of the tile's A2 buffer (it is dead before h1 is written).
+// Every wait is bounded: when a barrier does not complete in time the group records bit 0 in the status
+// word and skips its remaining steps; the CTA then frees its TMEM columns and returns.
 #include "sim_internal.h"
 #include "sim_envs.cuh"
 
 namespace simk {
 
-constexpr int kTcThreads = 128;
+constexpr int kTcThreads = 256;                   // per CTA
+constexpr uint32_t kTile = 128u;                  // envs (rows) per tile = threads per group
 constexpr uint32_t kTcLBO = 128u;                 // bytes between core matrices adjacent along K
-constexpr uint32_t kCh1 = 4u, kCh2 = 10u;         // 16-byte chunks per operand row: 16 TF32 values; 80 FP16 values
-constexpr uint32_t kTcCols = 64u;                 // TMEM columns (fp32): z1 / z2 use all, the logits the first 16
-// Instruction descriptors: D = fp32 (bit 4), A/B format (bits 7, 10: 2 = TF32, 0 = FP16), K-major, N >> 3 (bit 17), M >> 4 (bit 24).
-constexpr uint32_t kIdescTf32N64 = (1u << 4) | (2u << 7) | (2u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescF16N64 = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescF16N16 = (1u << 4) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kCh1 = 2u, kCh2 = 10u;         // 16-byte chunks per operand row: 16 and 80 FP16 values
+constexpr uint32_t kTileCols = 64u;               // TMEM columns (fp32) per tile: z1 / z2 use all, the logits the first 16
+constexpr uint32_t kTcCols = 2u * kTileCols;
+// Instruction descriptors: D = fp32 (bit 4), A = B = FP16 (0 at bits 7 and 10), K-major, N >> 3 (bit 17), M >> 4 (bit 24).
+constexpr uint32_t kIdescN64 = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescN16 = (1u << 4) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr long long kTcWaitCycles = 2000000000ll; // about a second at the SM clock
 
 struct TcSmem {
-    uint4 a1[128 * kCh1];   // layer-1 A operand (TF32 bit patterns)
-    uint4 a2[128 * kCh2];   // layer-2 / layer-3 A operand (FP16)
-    uint4 b1[64 * kCh1];    // layer-1 weights and bias (TF32, split)
-    uint4 b2[64 * kCh2];    // layer-2 weights and bias (FP16)
-    uint4 b3[16 * kCh2];    // layer-3 weights and bias (FP16, split), rows 4..15 zero
-    unsigned long long bar; // mbarrier the tensor core commits to
-    uint32_t tmem_slot;     // TMEM base address written by tcgen05.alloc
+    uint4 a[2][kTile * kCh2];  // per tile: A2 operand (FP16, 80 values per row); A1 (16 values per row) in its first 4 KB
+    uint4 b1[64 * kCh1];       // layer-1 weights and bias (split)
+    uint4 b2[64 * kCh2];       // layer-2 weights and bias
+    uint4 b3[16 * kCh2];       // layer-3 weights and bias (split), rows 4..15 zero
+    unsigned long long bar[2]; // per tile: mbarrier the tensor core commits to
+    uint32_t tmem_slot;        // TMEM base address written by tcgen05.alloc
 };
 
 struct TcCtx {
-    uint32_t tmem;
-    uint32_t parity;
+    uint32_t tmem;          // this group's accumulator columns, lane 0
+    uint32_t parity;        // phase parity of the group's mbarrier
+    uint32_t group;         // 0 or 1
+    uint32_t row;           // thread index inside the group
     bool fail;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t to_tf32(float x) { uint32_t r; asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x)); return r; }
-__device__ __forceinline__ float tf32_as_float(uint32_t u) { return __uint_as_float(u); }
 // f16x2 with `first` in the low half (the lower address / lower k).
 __device__ __forceinline__ uint32_t pack_f16x2(float first, float second) { uint32_t r; asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(second), "f"(first)); return r; }
 __device__ __forceinline__ uint32_t tanh_f16x2(uint32_t x) { uint32_t r; asm("tanh.approx.f16x2 %0, %1;" : "=r"(r) : "r"(x)); return r; }
 __device__ __forceinline__ uint16_t f16_bits(float x) { uint16_t r; asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(r) : "f"(x)); return r; }
 __device__ __forceinline__ float f16_value(uint16_t h) { float r; asm("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(h)); return r; }
+// x = hi + lo with hi = f16(x), lo = f16(x - hi).
+__device__ __forceinline__ void f16_split(float x, uint16_t &hi, uint16_t &lo) { hi = f16_bits(x); lo = f16_bits(__fsub_rn(x, f16_value(hi))); }
 
 // Shared-memory matrix descriptor: start address, leading and stride byte offsets (16-byte units),
 // descriptor version 1, no swizzle.
@@ -70,15 +76,26 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr, uint32_t chunks_per_
 // Index (in 16-byte chunks) of chunk c of row `row` of an operand tile with `ch` chunks per row.
 __device__ __forceinline__ uint32_t tc_chunk(uint32_t row, uint32_t c, uint32_t ch) { return (row >> 3) * ch * 8u + c * 8u + (row & 7u); }
 
-template <typename T>
-__device__ __forceinline__ void tc_put(uint4 *tile, uint32_t row, uint32_t k, uint32_t ch, T value)
+__device__ __forceinline__ void tc_put(uint4 *tile, uint32_t row, uint32_t k, uint32_t ch, uint16_t value)
 {
-    constexpr uint32_t per = 16u / sizeof(T);
-    reinterpret_cast<T *>(tile + tc_chunk(row, k / per, ch))[k % per] = value;
+    reinterpret_cast<uint16_t *>(tile + tc_chunk(row, k >> 3, ch))[k & 7u] = value;
 }
 
-// Stage the parameters as operand tiles, allocate the accumulator columns, initialise the barrier and the
-// constant columns of this thread's operand rows.  Called by all threads.
+// Group barrier (named barrier 1 + group, 128 threads) with an OR reduction of `flag`.
+__device__ __forceinline__ bool group_sync_or(uint32_t group, bool flag)
+{
+    uint32_t out;
+    if (group == 0u)
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(out) : "r"(flag ? 1u : 0u) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(out) : "r"(flag ? 1u : 0u) : "memory");
+    return out != 0u;
+}
+
+// Stage the parameters as operand tiles, allocate the accumulator columns, initialise the barriers.
+// Called by all threads of the CTA.
 __device__ __forceinline__ void tc_setup(const float *__restrict__ p, TcSmem &s, TcCtx &c)
 {
     const uint32_t tid = threadIdx.x;
@@ -86,33 +103,32 @@ __device__ __forceinline__ void tc_setup(const float *__restrict__ p, TcSmem &s,
     __syncthreads();
     for (uint32_t i = tid; i < 256u; i += kTcThreads) {               // W1[j][k]
         const uint32_t j = i >> 2, k = i & 3u;
-        const uint32_t hi = to_tf32(p[i]), lo = to_tf32(__fsub_rn(p[i], tf32_as_float(hi)));
-        tc_put<uint32_t>(s.b1, j, k, kCh1, hi); tc_put<uint32_t>(s.b1, j, 4u + k, kCh1, hi); tc_put<uint32_t>(s.b1, j, 8u + k, kCh1, lo);
+        uint16_t hi, lo;
+        f16_split(p[i], hi, lo);
+        tc_put(s.b1, j, k, kCh1, hi); tc_put(s.b1, j, 4u + k, kCh1, hi); tc_put(s.b1, j, 8u + k, kCh1, lo);
     }
     for (uint32_t j = tid; j < 64u; j += kTcThreads) {
-        const float b1 = p[256 + j], b2 = p[4416 + j];
-        const uint32_t hi = to_tf32(b1);
-        tc_put<uint32_t>(s.b1, j, 12u, kCh1, hi); tc_put<uint32_t>(s.b1, j, 13u, kCh1, to_tf32(__fsub_rn(b1, tf32_as_float(hi))));
-        const uint16_t h2 = f16_bits(b2);
-        tc_put<uint16_t>(s.b2, j, 64u, kCh2, h2); tc_put<uint16_t>(s.b2, j, 65u, kCh2, f16_bits(__fsub_rn(b2, f16_value(h2))));
+        uint16_t hi, lo;
+        f16_split(p[256 + j], hi, lo);
+        tc_put(s.b1, j, 12u, kCh1, hi); tc_put(s.b1, j, 13u, kCh1, lo);
+        f16_split(p[4416 + j], hi, lo);
+        tc_put(s.b2, j, 64u, kCh2, hi); tc_put(s.b2, j, 65u, kCh2, lo);
     }
-    for (uint32_t i = tid; i < 4096u; i += kTcThreads) tc_put<uint16_t>(s.b2, i >> 6, i & 63u, kCh2, f16_bits(p[320 + i]));
+    for (uint32_t i = tid; i < 4096u; i += kTcThreads) tc_put(s.b2, i >> 6, i & 63u, kCh2, f16_bits(p[320 + i]));
     for (uint32_t i = tid; i < 128u; i += kTcThreads) {               // W3[a][k] -> rows 2a (hi), 2a+1 (lo)
         const uint32_t a = i >> 6, k = i & 63u;
-        const uint16_t hi = f16_bits(p[4480 + i]);
-        tc_put<uint16_t>(s.b3, 2u * a, k, kCh2, hi); tc_put<uint16_t>(s.b3, 2u * a + 1u, k, kCh2, f16_bits(__fsub_rn(p[4480 + i], f16_value(hi))));
+        uint16_t hi, lo;
+        f16_split(p[4480 + i], hi, lo);
+        tc_put(s.b3, 2u * a, k, kCh2, hi); tc_put(s.b3, 2u * a + 1u, k, kCh2, lo);
     }
     if (tid < 2u) {
-        const float b3 = p[4608 + tid];
-        const uint16_t hi = f16_bits(b3);
-        tc_put<uint16_t>(s.b3, 2u * tid, 64u, kCh2, hi); tc_put<uint16_t>(s.b3, 2u * tid, 65u, kCh2, f16_bits(__fsub_rn(b3, f16_value(hi))));
+        uint16_t hi, lo;
+        f16_split(p[4608 + tid], hi, lo);
+        tc_put(s.b3, 2u * tid, 64u, kCh2, hi); tc_put(s.b3, 2u * tid, 65u, kCh2, lo);
     }
-    // constant columns of my rows: the two ones that multiply the bias parts, zero padding
-    s.a1[tc_chunk(tid, 3u, kCh1)] = make_uint4(0x3F800000u, 0x3F800000u, 0u, 0u);
-    s.a2[tc_chunk(tid, 8u, kCh2)] = make_uint4(0x3C003C00u, 0u, 0u, 0u);
-    s.a2[tc_chunk(tid, 9u, kCh2)] = make_uint4(0u, 0u, 0u, 0u);
     if (tid == 0u) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&s.bar)), "r"(1u) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&s.bar[0])), "r"(1u) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&s.bar[1])), "r"(1u) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < 32u) {
@@ -123,47 +139,51 @@ __device__ __forceinline__ void tc_setup(const float *__restrict__ p, TcSmem &s,
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    c.tmem = s.tmem_slot;
+    c.group = tid >> 7;
+    c.row = tid & 127u;
+    c.tmem = s.tmem_slot + c.group * kTileCols;
     c.parity = 0u;
     c.fail = false;
 }
 
-// Free the accumulator columns.  Called by all threads, after the last tc_policy.
-__device__ __forceinline__ void tc_teardown(TcCtx &c)
+// Free the accumulator columns.  Called by all threads of the CTA, after their last tc_policy.
+__device__ __forceinline__ void tc_teardown(TcSmem &s)
 {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x < 32)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(c.tmem), "r"(kTcCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s.tmem_slot), "r"(kTcCols) : "memory");
 }
 
-// One contraction D[128 x N] = A[128 x 16 nk bytes...] B^T over `nk` instructions of 32 bytes of K each (8 TF32 or
-// 16 FP16 values): publish this thread's operand row, let thread 0 issue, wait (bounded) for completion.
-// Returns false for the whole CTA when a wait ran out earlier; a wait that runs out now is reported by the next call.
-template <bool TF32>
-__device__ __forceinline__ bool tc_contract(uint32_t a_addr, uint32_t a_ch, uint32_t b_addr, uint32_t b_ch, uint32_t nk, uint32_t idesc,
-                                            TcSmem &s, TcCtx &c, uint32_t *status)
+enum : int { LAYER1 = 0, LAYER2 = 1, LAYER3 = 2 };
+
+// Publish the group's operand rows, let its first thread issue the contraction of `LAYER` and commit it to the
+// group's mbarrier, and wait (bounded) for completion.  Returns false for the whole group when a wait ran out
+// earlier; a wait that runs out now sets the status bit and is turned into the group-wide exit by the next call.
+template <int LAYER>
+__device__ __forceinline__ bool tc_contract(TcSmem &s, TcCtx &c, uint32_t *status)
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // my operand row: generic-proxy stores -> async proxy
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");  // my accumulator reads so far are done
-    if (__syncthreads_or(c.fail ? 1 : 0)) { c.fail = true; return false; }
-    if (threadIdx.x == 0) {
+    if (group_sync_or(c.group, c.fail)) { c.fail = true; return false; }
+    const uint32_t bar = smem_u32(&s.bar[c.group]);
+    if (c.row == 0u) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_u32(s.a[c.group]);
+        const uint32_t b_addr = LAYER == LAYER1 ? smem_u32(s.b1) : LAYER == LAYER2 ? smem_u32(s.b2) : smem_u32(s.b3);
+        constexpr uint32_t ch = LAYER == LAYER1 ? kCh1 : kCh2;
+        constexpr uint32_t nk = LAYER == LAYER1 ? 1u : 5u;           // instructions of K = 16 values (two core matrices) each
+        constexpr uint32_t idesc = LAYER == LAYER3 ? kIdescN16 : kIdescN64;
+#pragma unroll
         for (uint32_t k = 0; k < nk; ++k) {
-            const uint64_t da = tc_desc(a_addr + k * 2u * kTcLBO, a_ch), db = tc_desc(b_addr + k * 2u * kTcLBO, b_ch);
+            const uint64_t da = tc_desc(a_addr + k * 2u * kTcLBO, ch), db = tc_desc(b_addr + k * 2u * kTcLBO, ch);
             const uint32_t accumulate = k ? 1u : 0u;
-            if (TF32)
-                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                             "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-                             :: "r"(c.tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
-            else
-                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                             :: "r"(c.tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                         :: "r"(c.tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(smem_u32(&s.bar)) : "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
     }
-    const uint32_t bar = smem_u32(&s.bar);
     const long long t0 = clock64();
     uint32_t done = 0u;
     for (;;) {
@@ -177,7 +197,7 @@ __device__ __forceinline__ bool tc_contract(uint32_t a_addr, uint32_t a_ch, uint
     return true;
 }
 
-// Columns col0 .. col0+15 of this thread's accumulator row.
+// Columns 0..15 from `taddr` of this thread's accumulator row.
 __device__ __forceinline__ void tc_load16(uint32_t taddr, uint32_t (&v)[16])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -186,54 +206,62 @@ __device__ __forceinline__ void tc_load16(uint32_t taddr, uint32_t (&v)[16])
                  : "r"(taddr));
 }
 
-// My accumulator row (64 columns) -> tanh -> FP16 -> my row of the A2 tile.
-__device__ __forceinline__ void tc_activate(uint32_t taddr, TcSmem &s)
+// My accumulator row (64 columns) -> tanh -> FP16 -> my row of the group's A2 operand.
+__device__ __forceinline__ void tc_activate(TcSmem &s, const TcCtx &c)
 {
-    uint32_t v[4][16];
+    const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
+    uint4 *row = s.a[c.group] + tc_chunk(c.row, 0u, kCh2);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) tc_load16(taddr + 16u * (uint32_t)q, v[q]);
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-    uint4 *row = s.a2 + tc_chunk(threadIdx.x, 0u, kCh2);
+    for (int half = 0; half < 2; ++half) {
+        uint32_t v[2][16];
+        tc_load16(taddr + 32u * (uint32_t)half, v[0]);
+        tc_load16(taddr + 32u * (uint32_t)half + 16u, v[1]);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
+        for (int q = 0; q < 2; ++q)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            uint4 u;
-            u.x = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 0]), __uint_as_float(v[q][8 * h + 1])));
-            u.y = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 2]), __uint_as_float(v[q][8 * h + 3])));
-            u.z = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 4]), __uint_as_float(v[q][8 * h + 5])));
-            u.w = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 6]), __uint_as_float(v[q][8 * h + 7])));
-            row[(2 * q + h) * 8] = u;                                  // chunk 2q+h of my row
-        }
+            for (int h = 0; h < 2; ++h) {
+                uint4 u;
+                u.x = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 0]), __uint_as_float(v[q][8 * h + 1])));
+                u.y = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 2]), __uint_as_float(v[q][8 * h + 3])));
+                u.z = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 4]), __uint_as_float(v[q][8 * h + 5])));
+                u.w = tanh_f16x2(pack_f16x2(__uint_as_float(v[q][8 * h + 6]), __uint_as_float(v[q][8 * h + 7])));
+                row[(4 * half + 2 * q + h) * 8] = u;                   // chunk index along K
+            }
+    }
 }
 
-// Logits of this thread's observation; the CTA's 128 threads evaluate their 128 observations together.
-// Returns false for the whole CTA when a wait ran out.
+// Logits of this thread's observation; the group's 128 threads evaluate their 128 observations together.
+// Returns false for the whole group when a wait ran out.
 __device__ __forceinline__ bool tc_policy(const float4 o, TcSmem &s, TcCtx &c, uint32_t *status, f2 &logits)
 {
-    const uint32_t r = threadIdx.x;
-    const uint32_t taddr = c.tmem + ((r & ~31u) << 16);
-    {   // layer-1 operand row: observation split into two TF32 parts
-        const uint32_t h0 = to_tf32(o.x), h1 = to_tf32(o.y), h2 = to_tf32(o.z), h3 = to_tf32(o.w);
-        const uint4 hi = make_uint4(h0, h1, h2, h3);
-        const uint4 lo = make_uint4(to_tf32(__fsub_rn(o.x, tf32_as_float(h0))), to_tf32(__fsub_rn(o.y, tf32_as_float(h1))),
-                                    to_tf32(__fsub_rn(o.z, tf32_as_float(h2))), to_tf32(__fsub_rn(o.w, tf32_as_float(h3))));
-        uint4 *row = s.a1 + tc_chunk(r, 0u, kCh1);
-        row[0] = hi; row[8] = lo; row[16] = hi;
+    {   // layer-1 operand row: (o_hi[4], o_lo[4]) (o_hi[4], 1, 1, 0, 0)
+        const uint32_t h01 = pack_f16x2(o.x, o.y), h23 = pack_f16x2(o.z, o.w);
+        const float r0 = __fsub_rn(o.x, f16_value((uint16_t)(h01 & 0xFFFFu))), r1 = __fsub_rn(o.y, f16_value((uint16_t)(h01 >> 16)));
+        const float r2 = __fsub_rn(o.z, f16_value((uint16_t)(h23 & 0xFFFFu))), r3 = __fsub_rn(o.w, f16_value((uint16_t)(h23 >> 16)));
+        uint4 *row = s.a[c.group] + tc_chunk(c.row, 0u, kCh1);
+        row[0] = make_uint4(h01, h23, pack_f16x2(r0, r1), pack_f16x2(r2, r3));
+        row[8] = make_uint4(h01, h23, 0x3C003C00u, 0u);
     }
-    if (!tc_contract<true>(smem_u32(s.a1), kCh1, smem_u32(s.b1), kCh1, 2u, kIdescTf32N64, s, c, status)) return false;
-    tc_activate(taddr, s);
-    if (!tc_contract<false>(smem_u32(s.a2), kCh2, smem_u32(s.b2), kCh2, 5u, kIdescF16N64, s, c, status)) return false;
-    tc_activate(taddr, s);
-    if (!tc_contract<false>(smem_u32(s.a2), kCh2, smem_u32(s.b3), kCh2, 5u, kIdescF16N16, s, c, status)) return false;
+    if (!tc_contract<LAYER1>(s, c, status)) return false;
+    {   // the bias columns of my A2 row (the A1 rows of other threads may have covered them)
+        uint4 *row = s.a[c.group] + tc_chunk(c.row, 0u, kCh2);
+        row[8 * 8] = make_uint4(0x3C003C00u, 0u, 0u, 0u);
+        row[9 * 8] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    tc_activate(s, c);
+    if (!tc_contract<LAYER2>(s, c, status)) return false;
+    tc_activate(s, c);
+    if (!tc_contract<LAYER3>(s, c, status)) return false;
+    const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
     uint32_t l0, l1, l2, l3;
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(l0), "=r"(l1), "=r"(l2), "=r"(l3) : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
     logits = pk(__fadd_rn(__uint_as_float(l0), __uint_as_float(l1)), __fadd_rn(__uint_as_float(l2), __uint_as_float(l3)));
-    return true;                        // a wait that ran out just now is reported (CTA-wide) by the next contraction
+    return true;
 }
 
-__global__ void __launch_bounds__(kTcThreads, 5)
+__global__ void __launch_bounds__(kTcThreads, 4)
 rollout_cartpole_mlp_tc_kernel(const __grid_constant__ S4Args a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -241,7 +269,7 @@ rollout_cartpole_mlp_tc_kernel(const __grid_constant__ S4Args a)
     TcCtx ctx;
     tc_setup(a.params, ms, ctx);
 
-    // Every thread takes part in every barrier: threads past the batch shadow the last env and store nothing.
+    // Every thread takes part in every barrier of its group: threads past the batch shadow the last env and store nothing.
     const uint64_t i64 = (uint64_t)blockIdx.x * kTcThreads + threadIdx.x;
     const bool valid = i64 < a.n;
     const uint32_t i = valid ? (uint32_t)i64 : a.n - 1u;
@@ -278,10 +306,10 @@ rollout_cartpole_mlp_tc_kernel(const __grid_constant__ S4Args a)
         }
     }
     if (valid && ok) { a.state[i] = s; a.ep_len[i] = len; a.reset_count[i] = rc; }
-    tc_teardown(ctx);
+    tc_teardown(ms);
 }
 
-__global__ void __launch_bounds__(kTcThreads, 5)
+__global__ void __launch_bounds__(kTcThreads, 4)
 policy_logits_tc_kernel(const float4 *__restrict__ obs, int64_t M, const float *__restrict__ params, float2 *__restrict__ logits, uint32_t *status)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -293,7 +321,7 @@ policy_logits_tc_kernel(const float4 *__restrict__ obs, int64_t M, const float *
     f2 l;
     const bool ok = tc_policy(obs[valid ? i : M - 1], ms, ctx, status, l);
     if (valid && ok) logits[i] = make_float2(lo(l), hi(l));
-    tc_teardown(ctx);
+    tc_teardown(ms);
 }
 
 static cudaError_t tc_opt_in()
@@ -310,7 +338,7 @@ cudaError_t launch_cartpole_mlp_tc(const S4Args &a, cudaStream_t st)
 {
     cudaError_t e = tc_opt_in();
     if (e != cudaSuccess) return e;
-    const unsigned blocks = (a.n + kTcThreads - 1u) / kTcThreads;
+    const unsigned blocks = (unsigned)(((uint64_t)a.n + kTcThreads - 1u) / kTcThreads);
     rollout_cartpole_mlp_tc_kernel<<<blocks, kTcThreads, sizeof(TcSmem), st>>>(a);
     return cudaGetLastError();
 }
