@@ -28,6 +28,9 @@ if ROOT not in sys.path:
 from paper_2207_07736_b200 import inputs, shard  # noqa: E402
 
 FP32_LANES_PER_SM = 128
+XU_LANES_PER_SM = 16                      # special-function unit: measured 15.9 tanh.approx.f32 per clock and SM
+TANH_PER_ENV_STEP = 128
+TENSOR_FLOPS_PER_ENV_STEP = 2 * (16 * 64 + 80 * 64 + 80 * 16)   # the three padded contractions of the tensor-mode policy
 TRAJ_BYTES_S4 = 22          # obs 16 + act 1 + rew 4 + done 1
 # nominal / operation-expanded flops per env-step (fma = 2, any other fp32 op = 1, integer work = 0)
 FLOPS = {"cartpole": (27, 52), "acrobot": (181, 455), "mlp": (9094, 12205)}
@@ -293,7 +296,22 @@ def run_gpu(args, w):
     fp32_peak_tflops = 2 * FP32_LANES_PER_SM * sms * sm_max_mhz * 1e6 / 1e12
     t_hbm = bytes_per_env_step / (hbm_peak * 1e9)
     t_alu = fl_nom / (fp32_peak_tflops * 1e12)
-    if t_hbm >= t_alu:
+    if args.policy_mode == "tensor" and w.mlp_seed is not None:
+        # Tensor-mode policy: the matmuls are on the tensor cores, so the fp32 ledger no longer describes the
+        # kernel.  What binds it is the special-function unit (16 lanes per SM, one approximate tanh per lane
+        # and clock): 128 tanh evaluations per env-step.
+        xu_peak = XU_LANES_PER_SM * sms * sm_max_mhz * 1e6 / 1e12
+        achieved = TANH_PER_ENV_STEP * n * k_per_launch / (launch_ms * 1e-3) / 1e12
+        tensor_tflops = TENSOR_FLOPS_PER_ENV_STEP * n * k_per_launch / (launch_ms * 1e-3) / 1e12
+        bf16_peak = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))).get("bf16_tflops") if peak_kind == "measured" else 1590.0
+        roofline = {"bound": "alu", "achieved": achieved, "peak": xu_peak, "unit": "Tops/s", "frac": achieved / xu_peak,
+                    "traffic": args.traffic_bytes,
+                    "peak_source": "special-function unit: %d lanes x %d SMs x %.0f MHz (sm_max_mhz of MEASURED_PEAKS.json, of %s)" % (XU_LANES_PER_SM, sms, sm_max_mhz, peak_kind),
+                    "ops_ledger": "%d tanh per env-step (two hidden layers of 64 units)" % TANH_PER_ENV_STEP,
+                    "tensor": {"flops_per_env_step": TENSOR_FLOPS_PER_ENV_STEP, "achieved_tflops": tensor_tflops, "peak_tflops": bf16_peak,
+                               "frac": tensor_tflops / bf16_peak, "note": "FP16 tcgen05 contractions (padded shapes), against the measured dense bf16 peak"},
+                    "hbm_frac": bytes_per_launch / (launch_ms * 1e-3) / 1e9 / hbm_peak}
+    elif t_hbm >= t_alu:
         achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
                     "traffic": args.traffic_bytes, "peak_source": "MEASURED_PEAKS.json (of %s)" % peak_kind,

@@ -92,17 +92,19 @@ int sim_set_action_stream(sim_t *s, int mode);
  * sim_policy_logits (CartPole only; SIM_EINVAL for other env kinds or an unknown mode).
  *   SIM_POLICY_EXACT (default): the fp32 definition at the top of this file; actions are bit-reproducible.
  *   SIM_POLICY_TENSOR: tolerance mode for throughput (the fusion of simulation and inference that
- *     Section 7 of the paper leaves as future work, with the hidden layer on the tensor cores):
- *       h1 = tanh~(W1 obs + b1)            layer-1 sums as in exact mode; tanh~ = the GPU's approximate
- *                                          tanh instruction (relative error about 2^-11)
- *       z2 = b2 + sum_k tf32(W2[j][k]) * tf32(h1[k])   operands rounded to TF32 (10-bit mantissa,
- *                                          round to nearest, ties away), products exact, fp32 accumulation
- *                                          in the order the tensor core chooses
- *       h2 = tanh~(z2);  logits = b3 + W3 h2 in fp32, ascending j.
- *     Sampling, physics, reset and outputs are unchanged, so a trajectory stays an exact CartPole
- *     trajectory under the actions it records; only the action probabilities differ from exact mode,
- *     by the logit error (bounded by sum_j |W3[i][j]| (eps + sum_k |W2[j][k]| (eps + 2^-10)) with
- *     eps = 2^-10.9, far less for typical weights).  Not bit-reproducible across GPU generations.
+ *     Section 7 of the paper leaves as future work, with all three layers on the tensor cores):
+ *       z1 = W1 obs + b1      observation, W1 and b1 each split into two FP16 parts (x = hi + lo); the
+ *                             products hi*hi, lo*hi, hi*lo are exact and summed in fp32: about 21 bits
+ *       h1 = tanh~(f16(z1))   tanh~ = the GPU's packed half-precision tanh approximation (absolute error
+ *                             about 2^-11), result in FP16
+ *       z2 = b2 + sum_k f16(W2[j][k]) * h1[k]   FP16 operands (b2 split in two parts), products exact,
+ *                             fp32 accumulation in the order the tensor core chooses
+ *       h2 = tanh~(f16(z2));  logits = b3 + W3 h2 with W3 and b3 split in two FP16 parts, fp32 accumulation.
+ *     Parameters beyond the FP16 range (|x| > 65504) saturate.  Sampling, physics, reset and outputs are
+ *     unchanged, so a trajectory stays an exact CartPole trajectory under the actions it records; only the
+ *     action probabilities differ from exact mode, by the logit error, which is bounded by
+ *       sum_j |W3[i][j]| (e + sum_k |W2[j][k]| (e + 2^-11 |h1[k]|)),  e = 2^-10.987 + 0.448 * 2^-11,
+ *     and is far smaller for typical weights.  Not bit-reproducible across GPU generations.
  * The first call that selects tensor mode allocates a 4-byte device status word (see
  * sim_get_device_status). */
 enum { SIM_POLICY_EXACT = 0, SIM_POLICY_TENSOR = 1 };
