@@ -184,12 +184,15 @@ __device__ __forceinline__ bool tc_contract(TcSmem &s, TcCtx &c, uint32_t *statu
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
     }
-    const long long t0 = clock64();
     uint32_t done = 0u;
-    for (;;) {
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(c.parity) : "memory");
-        if (done || clock64() - t0 > kTcWaitCycles) break;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(c.parity) : "memory");
+    if (!done) {                                                       // rare: the first wait timed out inside the hardware
+        const long long t0 = clock64();
+        do {
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                         : "=r"(done) : "r"(bar), "r"(c.parity) : "memory");
+        } while (!done && clock64() - t0 <= kTcWaitCycles);
     }
     if (!done) { c.fail = true; if (status) atomicOr(status, 1u); }
     c.parity ^= 1u;
