@@ -188,3 +188,31 @@ def test_cfg3_full_size_in_tensor_mode():
     ref = exact.rollout(20, 20, torch.from_numpy(p).cuda(), want=("act",))
     f_t = float((out["act"][:20] == 0).float().mean()); f_e = float((ref["act"] == 0).float().mean())
     assert abs(f_t - f_e) < 2e-3, (f_t, f_e)
+
+
+@pytest.mark.parametrize("n", [1, 129, 257])
+def test_tensor_rollout_tiny_and_ragged_batches(n):
+    """One env (a CTA whose second group only shadows), one env past a tile, one env past a CTA."""
+    torch = torch_cuda()
+    T, seed = 30, 8
+    p = inputs.mlp_params(5, 0.2)
+    sim = binding.Sim(oracle.CARTPOLE, n, 4, seed, policy_mode=binding.SIM_POLICY_TENSOR)
+    out = sim.rollout(T, 4, torch.from_numpy(p).cuda())           # 8 launches, the last one of 2 steps
+    torch.cuda.synchronize()
+    assert sim.device_status() == 0 and sim.launches == 1 + 8
+    check_tensor_rollout(sim, out, p, seed, np.arange(n, dtype=np.uint32), T, "tiny n%d" % n)
+
+
+def test_tensor_mode_leaves_buffers_alone_and_handles_null_outputs():
+    torch = torch_cuda()
+    n, T, seed = 200, 12, 2
+    p = torch.from_numpy(inputs.mlp_params(1)).cuda()
+    a = binding.Sim(oracle.CARTPOLE, n, 4, seed, policy_mode=binding.SIM_POLICY_TENSOR)
+    full = a.rollout(T, T, p)
+    b = binding.Sim(oracle.CARTPOLE, n, 4, seed, policy_mode=binding.SIM_POLICY_TENSOR)
+    guard = torch.full((T * n + 64,), 7, dtype=torch.uint8, device="cuda")
+    binding.sim_rollout(b.h, T, 5, p, None, None, None, guard[32:32 + T * n])       # only the done flags
+    torch.cuda.synchronize()
+    assert bool((guard[:32] == 7).all()) and bool((guard[32 + T * n:] == 7).all())
+    assert torch.equal(guard[32:32 + T * n].view(T, n), full["done"])
+    assert torch.equal(a.state(), b.state())
