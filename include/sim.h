@@ -117,6 +117,14 @@ int sim_set_policy_mode(sim_t *s, int mode);
 enum { SIM_STATUS_TENSOR_WAIT = 1 };
 int sim_get_device_status(sim_t *s, uint32_t *h_flags);
 
+/* sim_selfcheck_tensor_wait -- exercises the bounded wait of the tensor-mode kernels without a fault: one CTA
+ * runs the policy with its tensor-core contractions left out, so every wait must give up (after about a
+ * millisecond here), raise the status bit, skip the rest and free its tensor memory.  Synchronises the stream.
+ *   h_status            HOST: the status word of that launch (expected SIM_STATUS_TENSOR_WAIT)
+ *   h_threads_completed HOST: threads whose policy evaluation reported success (expected 0)
+ * Uses a status word of its own: the handle's status (sim_get_device_status) is not touched. */
+int sim_selfcheck_tensor_wait(sim_t *s, uint32_t *h_status, uint32_t *h_threads_completed);
+
 /* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env. */
 int sim_reset(sim_t *s);
 

@@ -27,6 +27,7 @@ SIGNATURES = {
     "sim_set_action_stream": (C.c_int, [C.c_void_p, C.c_int]),
     "sim_set_policy_mode": (C.c_int, [C.c_void_p, C.c_int]),
     "sim_get_device_status": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint32)]),
+    "sim_selfcheck_tensor_wait": (C.c_int, [C.c_void_p, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]),
     "sim_reset": (C.c_int, [C.c_void_p]),
     "sim_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "sim_rollout": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -130,6 +131,13 @@ def sim_get_device_status(h) -> int:
     flags = C.c_uint32(0)
     _check(lib().sim_get_device_status(h, C.byref(flags)), h)
     return flags.value
+
+
+def sim_selfcheck_tensor_wait(h):
+    """(status word, threads that reported success) of the bounded-wait self-check launch."""
+    status, completed = C.c_uint32(0), C.c_uint32(0)
+    _check(lib().sim_selfcheck_tensor_wait(h, C.byref(status), C.byref(completed)), h)
+    return status.value, completed.value
 
 
 def sim_reset(h):

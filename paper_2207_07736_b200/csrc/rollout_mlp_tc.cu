@@ -160,14 +160,15 @@ enum : int { LAYER1 = 0, LAYER2 = 1, LAYER3 = 2 };
 // Publish the group's operand rows, let its first thread issue the contraction of `LAYER` and commit it to the
 // group's mbarrier, and wait (bounded) for completion.  Returns false for the whole group when a wait ran out
 // earlier; a wait that runs out now sets the status bit and is turned into the group-wide exit by the next call.
-template <int LAYER>
-__device__ __forceinline__ bool tc_contract(TcSmem &s, TcCtx &c, uint32_t *status)
+// ISSUE = false (self-check only) leaves the contraction out, so that the wait must run out.
+template <int LAYER, bool ISSUE = true>
+__device__ __forceinline__ bool tc_contract(TcSmem &s, TcCtx &c, uint32_t *status, long long wait_cycles = kTcWaitCycles)
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // my operand row: generic-proxy stores -> async proxy
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");  // my accumulator reads so far are done
     if (group_sync_or(c.group, c.fail)) { c.fail = true; return false; }
     const uint32_t bar = smem_u32(&s.bar[c.group]);
-    if (c.row == 0u) {
+    if (ISSUE && c.row == 0u) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = smem_u32(s.a[c.group]);
         const uint32_t b_addr = LAYER == LAYER1 ? smem_u32(s.b1) : LAYER == LAYER2 ? smem_u32(s.b2) : smem_u32(s.b3);
@@ -192,7 +193,7 @@ __device__ __forceinline__ bool tc_contract(TcSmem &s, TcCtx &c, uint32_t *statu
         do {
             asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(done) : "r"(bar), "r"(c.parity) : "memory");
-        } while (!done && clock64() - t0 <= kTcWaitCycles);
+        } while (!done && clock64() - t0 <= wait_cycles);
     }
     if (!done) { c.fail = true; if (status) atomicOr(status, 1u); }
     c.parity ^= 1u;
@@ -236,7 +237,8 @@ __device__ __forceinline__ void tc_activate(TcSmem &s, const TcCtx &c)
 
 // Logits of this thread's observation; the group's 128 threads evaluate their 128 observations together.
 // Returns false for the whole group when a wait ran out.
-__device__ __forceinline__ bool tc_policy(const float4 o, TcSmem &s, TcCtx &c, uint32_t *status, f2 &logits)
+template <bool ISSUE = true>
+__device__ __forceinline__ bool tc_policy(const float4 o, TcSmem &s, TcCtx &c, uint32_t *status, f2 &logits, long long wait_cycles = kTcWaitCycles)
 {
     {   // layer-1 operand row: (o_hi[4], o_lo[4]) (o_hi[4], 1, 1, 0, 0)
         const uint32_t h01 = pack_f16x2(o.x, o.y), h23 = pack_f16x2(o.z, o.w);
@@ -246,16 +248,16 @@ __device__ __forceinline__ bool tc_policy(const float4 o, TcSmem &s, TcCtx &c, u
         row[0] = make_uint4(h01, h23, pack_f16x2(r0, r1), pack_f16x2(r2, r3));
         row[8] = make_uint4(h01, h23, 0x3C003C00u, 0u);
     }
-    if (!tc_contract<LAYER1>(s, c, status)) return false;
+    if (!tc_contract<LAYER1, ISSUE>(s, c, status, wait_cycles)) return false;
     {   // the bias columns of my A2 row (the A1 rows of other threads may have covered them)
         uint4 *row = s.a[c.group] + tc_chunk(c.row, 0u, kCh2);
         row[8 * 8] = make_uint4(0x3C003C00u, 0u, 0u, 0u);
         row[9 * 8] = make_uint4(0u, 0u, 0u, 0u);
     }
     tc_activate(s, c);
-    if (!tc_contract<LAYER2>(s, c, status)) return false;
+    if (!tc_contract<LAYER2, ISSUE>(s, c, status, wait_cycles)) return false;
     tc_activate(s, c);
-    if (!tc_contract<LAYER3>(s, c, status)) return false;
+    if (!tc_contract<LAYER3, ISSUE>(s, c, status, wait_cycles)) return false;
     const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
     uint32_t l0, l1, l2, l3;
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(l0), "=r"(l1), "=r"(l2), "=r"(l3) : "r"(taddr));
@@ -327,11 +329,28 @@ policy_logits_tc_kernel(const float4 *__restrict__ obs, int64_t M, const float *
     tc_teardown(ms);
 }
 
+// Self-check of the bounded wait: one CTA runs the policy with the contractions left out, so the first wait of
+// either group must run out (after `wait_cycles`), set the status bit and turn the next contraction into the
+// group-wide exit.  completed[i] = 1 if thread i's policy call reported success (expected: none).
+__global__ void __launch_bounds__(kTcThreads, 4)
+tensor_wait_selfcheck_kernel(const float *__restrict__ params, long long wait_cycles, uint32_t *status, uint32_t *completed)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TcSmem &ms = *reinterpret_cast<TcSmem *>(smem_raw);
+    TcCtx ctx;
+    tc_setup(params, ms, ctx);
+    f2 l;
+    const bool ok = tc_policy<false>(make_float4(0.0f, 0.0f, 0.0f, 0.0f), ms, ctx, status, l, wait_cycles);
+    completed[threadIdx.x] = ok ? 1u : 0u;
+    tc_teardown(ms);
+}
+
 static cudaError_t tc_opt_in()
 {
     static cudaError_t once = [] {
         cudaError_t e = cudaFuncSetAttribute(rollout_cartpole_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
         if (e == cudaSuccess) e = cudaFuncSetAttribute(policy_logits_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tensor_wait_selfcheck_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
         return e;
     }();
     return once;
@@ -355,6 +374,14 @@ cudaError_t launch_policy_logits_tc(const float *obs, int64_t M, const float *pa
     if (blocks > 0x7FFFFFFFll) return cudaErrorInvalidConfiguration;
     policy_logits_tc_kernel<<<(unsigned)blocks, kTcThreads, sizeof(TcSmem), st>>>(reinterpret_cast<const float4 *>(obs), M, params,
                                                                                   reinterpret_cast<float2 *>(logits), status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tensor_wait_selfcheck(const float *params, long long wait_cycles, uint32_t *status, uint32_t *completed, cudaStream_t st)
+{
+    cudaError_t e = tc_opt_in();
+    if (e != cudaSuccess) return e;
+    tensor_wait_selfcheck_kernel<<<1, kTcThreads, sizeof(TcSmem), st>>>(params, wait_cycles, status, completed);
     return cudaGetLastError();
 }
 

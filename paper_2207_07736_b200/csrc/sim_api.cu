@@ -391,6 +391,29 @@ SIM_API int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_misma
     return SIM_OK;
 }
 
+// One CTA of the tensor-mode policy with its contractions left out: every wait must give up after about a
+// millisecond.  Scratch: 4610 zero parameters, a status word and one word per thread.
+SIM_API int sim_selfcheck_tensor_wait(sim_t *s, uint32_t *h_status, uint32_t *h_threads_completed)
+{
+    if (!s || !h_status || !h_threads_completed) return SIM_EINVAL;
+    const size_t words = SIM_POLICY_PARAM_COUNT + 1 + 256;
+    uint32_t *d = nullptr;
+    CU(s, cudaMalloc(&d, words * sizeof(uint32_t)));
+    uint32_t h[257] = {0};
+    cudaError_t e = cudaMemsetAsync(d, 0, words * sizeof(uint32_t), s->stream);
+    if (e == cudaSuccess) e = launch_tensor_wait_selfcheck(reinterpret_cast<const float *>(d), 2000000ll, d + SIM_POLICY_PARAM_COUNT, d + SIM_POLICY_PARAM_COUNT + 1, s->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h, d + SIM_POLICY_PARAM_COUNT, sizeof(h), cudaMemcpyDeviceToHost, s->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+    cudaFree(d);
+    if (e != cudaSuccess) return cuda_fail(s, e);
+    s->launches += 1;
+    *h_status = h[0];
+    uint32_t done = 0;
+    for (int i = 0; i < 256; ++i) done += h[1 + i];
+    *h_threads_completed = done;
+    return SIM_OK;
+}
+
 SIM_API int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, float *d_obs6)
 {
     if (!s || !d_state || !d_obs6 || M < 0) return SIM_EINVAL;

@@ -86,6 +86,7 @@ cudaError_t launch_acrobot_random(const S4Args &a, cudaStream_t st);    // Acrob
 cudaError_t launch_cartpole_mlp(const S4Args &a, cudaStream_t st);      // CartPole, MLP policy, packed two-env kernel
 cudaError_t launch_cartpole_mlp_tc(const S4Args &a, cudaStream_t st);   // CartPole, MLP policy in tensor mode (tcgen05 hidden layer)
 cudaError_t launch_policy_logits_tc(const float *obs, int64_t M, const float *params, float *logits, uint32_t *status, cudaStream_t st);
+cudaError_t launch_tensor_wait_selfcheck(const float *params, long long wait_cycles, uint32_t *status, uint32_t *completed, cudaStream_t st);   // 256 words
 cudaError_t launch_division_selfcheck(int nums_per_den, unsigned long long *d_bad, cudaStream_t st);
 cudaError_t launch_synth(int S, const SynthArgs &a, cudaStream_t st);
 cudaError_t launch_acrobot_observation(const float *state, int64_t M, float *obs6, cudaStream_t st);

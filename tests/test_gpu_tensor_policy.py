@@ -216,3 +216,19 @@ def test_tensor_mode_leaves_buffers_alone_and_handles_null_outputs():
     assert bool((guard[:32] == 7).all()) and bool((guard[32 + T * n:] == 7).all())
     assert torch.equal(guard[32:32 + T * n].view(T, n), full["done"])
     assert torch.equal(a.state(), b.state())
+
+
+def test_bounded_wait_gives_up_cleanly():
+    """The tensor-mode kernels never spin without a limit: with the contractions left out (self-check launch)
+    every wait runs out, the status bit is raised, no thread reports success, tensor memory is freed, and the
+    context stays usable for an ordinary tensor-mode rollout afterwards."""
+    torch = torch_cuda()
+    sim = binding.Sim(oracle.CARTPOLE, 300, 4, 4, policy_mode=binding.SIM_POLICY_TENSOR)
+    status, completed = binding.sim_selfcheck_tensor_wait(sim.h)
+    assert status == binding.SIM_STATUS_TENSOR_WAIT and completed == 0
+    assert sim.device_status() == 0                       # the self-check has a status word of its own
+    p = inputs.mlp_params(1)
+    out = sim.rollout(16, 16, torch.from_numpy(p).cuda())
+    torch.cuda.synchronize()
+    assert sim.device_status() == 0
+    check_tensor_rollout(sim, out, p, 4, np.arange(300, dtype=np.uint32), 16, "after self-check")
