@@ -206,10 +206,12 @@ def run_reference(args, w):
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 def time_rollouts(torch, sim, w, K, reps, d_params, out):
-    """Device time (ms) of `reps` rollouts, each bracketed by its own pair of events on the sim's stream."""
+    """Device time (ms) of `reps` rollouts, each from a fresh (untimed) reset and bracketed by its own pair of
+    events on the sim's stream."""
     times = []
     for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sim.reset()
         e0.record()
         sim.rollout(w.T, K, d_params, out=out)
         e1.record()
@@ -331,11 +333,11 @@ def run_gpu(args, w):
     sweep = {}
     if not args.no_sweep:
         for k in w.k_sweep:
-            reps = max(3, min(args.steps, 10))
+            reps = max(5, min(args.steps, 10))
             time_rollouts(torch, sim, w, k, 1, d_params, out)
             ts = time_rollouts(torch, sim, w, k, reps, d_params, out)
             med = statistics.median(ts)
-            sweep[str(k)] = {"env_steps_per_sec": n * w.T / (med * 1e-3), "ms": med, "launches": -(-w.T // k),
+            sweep[str(k)] = {"env_steps_per_sec": n * w.T / (med * 1e-3), "ms": med, "ms_min": min(ts), "reps": reps, "launches": -(-w.T // k),
                              "bytes_per_env_step": algorithmic_bytes_per_env_step(w, k)}
         base = sweep.get("1")
         if base:
