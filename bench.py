@@ -37,6 +37,9 @@ FLOPS = {"cartpole": (27, 52), "acrobot": (181, 455), "mlp": (9094, 12205)}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused rollout kernel, from the ncu
 # captures summarised under profiles/ (keyed by workload and K_fused; other shapes report null)
 NCU_TRAFFIC_BYTES = {("cfg2", 1000): 1.3869e9}
+# tensor-mode policy: captured on a reduced cfg3 (N = 262 144, T = 100: 533.19 MB for 2.62e7 env-steps) and scaled
+# to the full launch by env-steps (the traffic is the trajectory, proportional to env-steps)
+NCU_TRAFFIC_BYTES_TENSOR = {("cfg3", 500): 533.19e6 / 2.62144e7 * (1048576 * 500)}
 
 
 def algorithmic_bytes_per_env_step(w, K):
@@ -325,7 +328,9 @@ def run_gpu(args, w):
                     "flops_ledger": "nominal %d flop/env-step (operation-expanded: %d)" % (fl_nom, fl_exp),
                     "frac_expanded_ledger": fl_exp * n * k_per_launch / (launch_ms * 1e-3) / 1e12 / fp32_peak_tflops}
     if roofline["traffic"] is None:
-        roofline["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, K))
+        table = NCU_TRAFFIC_BYTES_TENSOR if (args.policy_mode == "tensor" and w.mlp_seed is not None) else NCU_TRAFFIC_BYTES
+        full = inputs.WORKLOADS.get(w.name)                          # None for a reduced (profiling) shape
+        roofline["traffic"] = table.get((w.name, K)) if full is not None and n == full.n_envs and w.T == full.T else None
     roofline["kernel"] = "fused rollout kernel, K_fused=%d, %d launch(es) per step" % (K, launches_per_step)
     roofline["launch_ms"] = launch_ms
 
