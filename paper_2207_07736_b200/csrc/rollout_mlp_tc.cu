@@ -345,15 +345,19 @@ tensor_wait_selfcheck_kernel(const float *__restrict__ params, long long wait_cy
     tc_teardown(ms);
 }
 
+// The kernels need more than 48 KB of dynamic shared memory: opt in once per device.
 static cudaError_t tc_opt_in()
 {
-    static cudaError_t once = [] {
-        cudaError_t e = cudaFuncSetAttribute(rollout_cartpole_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(policy_logits_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tensor_wait_selfcheck_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
-        return e;
-    }();
-    return once;
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(rollout_cartpole_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(policy_logits_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tensor_wait_selfcheck_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
 }
 
 cudaError_t launch_cartpole_mlp_tc(const S4Args &a, cudaStream_t st)
