@@ -55,7 +55,12 @@ def test_argument_errors_are_host_side(L):
     for fn, args in [("sim_destroy", (None,)), ("sim_reset", (None,)), ("sim_set_stream", (None, None)),
                      ("sim_step", (None, None, None, None, None)), ("sim_get_state", (None, None)),
                      ("sim_rollout", (None, 1, 1, None, None, None, None, None)),
-                     ("sim_rollout_host", (None, 1, 1, None, None, None, None, None))]:
+                     ("sim_rollout_host", (None, 1, 1, None, None, None, None, None)),
+                     ("sim_set_policy_mode", (None, 1)), ("sim_get_device_status", (None, None)),
+                     ("sim_selfcheck_tensor_wait", (None, None, None)), ("sim_set_action_stream", (None, 0)),
+                     ("sim_set_compute_factor", (None, 1)), ("sim_set_env_offset", (None, 0)),
+                     ("sim_episode_returns", (None, None, None, 1, 1, None, None)),
+                     ("sim_acrobot_observation", (None, None, 1, None)), ("sim_policy_logits", (None, None, 1, None, None))]:
         assert getattr(L, fn)(*args) == EINVAL
     assert L.sim_launch_count(None) == -1 and L.sim_last_cuda_error(None) == 0
     for code in (0, -1, -2, -3, -4, -99):
