@@ -107,9 +107,10 @@ rollout_acrobot_x2_kernel(const __grid_constant__ S4Args a)
     const float PI = fbits(0x40490FDBu), W1M = fbits(0x41490FDBu), W2M = fbits(0x41E231D6u);
 
     const int nblk = (a.phase + a.K + 3) >> 2;
+    const PhiloxEnv pe_a = philox_prepare(env_a, a.rk), pe_b = philox_prepare(env_b, a.rk);
     for (int b = 0; b < nblk; ++b) {
-        const uint4 ba = philox(env_a, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
-        const uint4 bb = philox(env_b, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
+        const uint4 ba = philox_action_block(pe_a, a.tb0 + (uint32_t)b, a.rk);
+        const uint4 bb = philox_action_block(pe_b, a.tb0 + (uint32_t)b, a.rk);
 #pragma unroll 1
         for (int j = 0; j < 4; ++j) {
             const int k = 4 * b + j - a.phase;

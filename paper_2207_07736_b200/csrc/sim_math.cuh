@@ -33,6 +33,42 @@ __device__ __forceinline__ uint4 philox(uint32_t c0, uint32_t c1, uint32_t c2, u
     return make_uint4(c0, c1, c2, c3);
 }
 
+// The action blocks of one env have the counter (env, tb, 0, 0) with only tb changing, so everything in the
+// first three rounds that depends on the env and the keys alone is computed once per env (three of the six
+// multiplications of those rounds); philox_action_block(prepared, tb) == philox(env, tb, 0, 0).
+struct PhiloxEnv { uint32_t a, b, c, g; };
+
+__device__ __forceinline__ PhiloxEnv philox_prepare(uint32_t env, const RoundKeys &rk)
+{
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t e2 = __umulhi(M0, env) ^ rk.k[0][1], e3 = M0 * env;      // state after round 0: (tb ^ k00, 0, e2, e3)
+    const uint32_t f0 = __umulhi(M1, e2) ^ rk.k[1][0], f1 = M1 * e2;        // after round 1: (f0, f1, hi(M0 x) ^ e3 ^ k11, lo(M0 x))
+    PhiloxEnv p;
+    p.a = e3 ^ rk.k[1][1];
+    p.b = f1 ^ rk.k[2][0];
+    p.c = __umulhi(M0, f0) ^ rk.k[2][1];
+    p.g = M0 * f0;
+    return p;
+}
+
+__device__ __forceinline__ uint4 philox_action_block(const PhiloxEnv &p, uint32_t tb, const RoundKeys &rk)
+{
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t x = tb ^ rk.k[0][0];
+    uint32_t c2 = __umulhi(M0, x) ^ p.a, c3 = M0 * x;                        // round 1
+    uint32_t c0 = __umulhi(M1, c2) ^ p.b, c1 = M1 * c2;                      // round 2
+    c2 = c3 ^ p.c; c3 = p.g;
+#pragma unroll
+    for (int r = 3; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+        uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        uint32_t n0 = hi1 ^ c1 ^ rk.k[r][0];
+        uint32_t n2 = hi0 ^ c3 ^ rk.k[r][1];
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
 // u in [0, 1 - 2^-24]: top 24 bits, exact.
 __device__ __forceinline__ float uniform01(uint32_t w) { return __fmul_rn(__uint2float_rn(w >> 8), fbits(0x33800000u)); }
 
