@@ -36,7 +36,7 @@ TRAJ_BYTES_S4 = 22          # obs 16 + act 1 + rew 4 + done 1
 FLOPS = {"cartpole": (27, 52), "acrobot": (181, 455), "mlp": (9094, 12205)}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused rollout kernel, from the ncu
 # captures summarised under profiles/ (keyed by workload and K_fused; other shapes report null)
-NCU_TRAFFIC_BYTES = {("cfg2", 1000): 1.3869e9}
+NCU_TRAFFIC_BYTES = {("cfg2", 1000): 1.3863e9}
 # tensor-mode policy: captured on a reduced cfg3 (N = 262 144, T = 100: 533.19 MB for 2.62e7 env-steps) and scaled
 # to the full launch by env-steps (the traffic is the trajectory, proportional to env-steps)
 NCU_TRAFFIC_BYTES_TENSOR = {("cfg3", 500): 533.19e6 / 2.62144e7 * (1048576 * 500)}
