@@ -18,6 +18,8 @@
  *     reset_count [N] u32) are owned by the library: sim_create allocates, sim_destroy frees.
  *   - Except sim_create / sim_destroy / sim_rollout_host, calls only enqueue work on the
  *     handle's stream and return; the caller synchronises the stream.
+ *   - A handle belongs to the CUDA device that was current in sim_create; a call made while
+ *     another device is current returns SIM_ESTATE and enqueues nothing.
  *   - All floating point is IEEE binary32 with a fixed operation order, so results are
  *     reproducible bit for bit for a given (seed, env index, step index), whatever K is.
  *   - Random numbers: Philox4x32-10 keyed by the seed.  Action word of (env, t) = word
@@ -45,9 +47,9 @@ enum { SIM_OK = 0, SIM_EINVAL = -1, SIM_ENOMEM = -2, SIM_ECUDA = -3, SIM_ESTATE 
 #define SIM_POLICY_PARAM_COUNT 4610   /* W1[64][4] b1[64] W2[64][64] b2[64] W3[2][64] b3[2], rows = output units */
 
 /*
- * sim_create -- make N simulator instances on the current CUDA device (Section 3: "N
- * simulator instances in parallel"; Section 2.2: CartPole state of S = 4 floats; Section
- * 4.2: the state-size factor S of the synthetic simulator).
+ * sim_create -- make N simulator instances on the current CUDA device (Section 3: the N
+ * parallel simulator instances of GPU vectorization; Section 2.2: the CartPole state of S = 4
+ * floats; Section 4.2: the state-size factor S of the synthetic simulator).
  *   out       receives the handle.
  *   env_kind  SIM_CARTPOLE | SIM_ACROBOT | SIM_SYNTH.
  *   n_envs    1 .. 2^32-1.
@@ -58,20 +60,25 @@ enum { SIM_OK = 0, SIM_EINVAL = -1, SIM_ENOMEM = -2, SIM_ECUDA = -3, SIM_ESTATE 
  */
 int sim_create(sim_t **out, int env_kind, int64_t n_envs, int state_dim, uint64_t seed);
 
-/* sim_destroy -- wait for the handle's stream, free everything.  NULL is SIM_EINVAL. */
+/* sim_destroy -- wait for the handle's stream, free everything.  NULL is SIM_EINVAL.
+ * (No passage of the paper: lifetime hook.) */
 int sim_destroy(sim_t *s);
 
-/* sim_set_stream -- use this cudaStream_t (passed as void*) for all later work; NULL = default stream. */
+/* sim_set_stream -- use this cudaStream_t (passed as void*) for all later work; NULL = default stream.
+ * (No passage of the paper: plumbing hook; the stream belongs to the caller.) */
 int sim_set_stream(sim_t *s, void *cuda_stream);
 
 /* sim_set_env_offset -- global index of this handle's env 0 (default 0).  Random draws are keyed by
  * offset + local index, so handles that own disjoint ranges of one global population reproduce the
  * single-handle result exactly (sharding across GPUs needs no exchange: envs never interact).
- * offset + n_envs must not exceed 2^32.  Takes effect at the next sim_reset. */
+ * offset + n_envs must not exceed 2^32.  Action draws use the new offset from the next call on, reset
+ * draws from the next reset on; the states a handle already holds were drawn with the old offset, so call
+ * sim_reset after changing it.  (No passage of the paper: Section 3 only says the instances are independent,
+ * which is what makes this sharding exact.) */
 int sim_set_env_offset(sim_t *s, uint64_t env_offset);
 
-/* sim_set_compute_factor -- the paper's compute-factor knob C (Section 4.2, "increases the compute
- * requirements ... by increasing the number of simulation iterations"): one recorded step becomes C
+/* sim_set_compute_factor -- the paper's compute-factor knob C (Section 4.2: C multiplies the number of
+ * simulation iterations per step, and with it the compute per step): one recorded step becomes C
  * iterations of the env's dynamics update under the step's one action (for Acrobot each iteration is a
  * full RK4 step with wrap and clip); reward, the done test and ep_len refer to the state after the last
  * iteration, and the trajectory still has one row per recorded step.  1 <= C <= 65536, default 1 (the
@@ -89,10 +96,23 @@ enum { SIM_ACTIONS_WORD = 0, SIM_ACTIONS_BITS = 1 };
 int sim_set_action_stream(sim_t *s, int mode);
 
 /* sim_set_policy_mode -- how the MLP policy is evaluated inside sim_rollout / sim_rollout_host /
- * sim_policy_logits (CartPole only; SIM_EINVAL for other env kinds or an unknown mode).
- *   SIM_POLICY_EXACT (default): the fp32 definition at the top of this file; actions are bit-reproducible.
- *   SIM_POLICY_TENSOR: tolerance mode for throughput (the fusion of simulation and inference that
- *     Section 7 of the paper leaves as future work, with all three layers on the tensor cores):
+ * sim_policy_logits (CartPole only; SIM_EINVAL for other env kinds or an unknown mode).  The two tensor modes are
+ * the fusion of simulation and inference that Section 7 of the paper leaves as future work, with all three layers
+ * on the tensor cores; the arithmetic is this library's.  Which mode meets which tolerance:
+ *   SIM_POLICY_EXACT (default): the fp32 definition at the top of this file.  Logits, actions and everything
+ *     else are bit-reproducible (tolerance: none).
+ *   SIM_POLICY_TENSOR_PRECISE: logits within 1e-5 (absolute) of the fp32 definition for weights and observations
+ *     of ordinary size (checked up to logits of magnitude 7); a sampled action can differ from exact mode only where
+ *     the uniform draw lies within the resulting change of the action probability (below 1e-5 of the env-steps).
+ *       z1 = W1 obs + b1      observation, W1 and b1 each split into THREE FP16 parts (x = x1 + x2 + x3); the six
+ *                             leading products of parts are exact and summed in fp32 by the tensor core
+ *       h1 = tanh'(z1)        tanh'(z) = 1 - 2 / (2^(2 log2(e) z) + 1) in fp32 with the GPU's base-2 exponential
+ *                             and reciprocal approximations: absolute error below 3e-7
+ *       z2 = b2 + W2 h1       h1 = hi + lo (hi = h1 cut to 11 significant bits, lo = f16(h1 - hi)), W2 = f16(W2) +
+ *                             f16(W2 - f16(W2)); hi*hi + hi*lo + lo*hi summed in fp32 by the tensor core, b2 added in fp32
+ *       h2 = tanh'(z2);       logits = b3 + W3 h2 with the same splits.
+ *   SIM_POLICY_TENSOR: the fast mode; it does NOT meet the 1e-5 logit tolerance (typical logit error 2e-3, bound
+ *     below); use it where throughput matters more than the third digit of the action probabilities.
  *       z1 = W1 obs + b1      observation, W1 and b1 each split into two FP16 parts (x = hi + lo); the
  *                             products hi*hi, lo*hi, hi*lo are exact and summed in fp32: about 21 bits
  *       h1 = tanh~(f16(z1))   tanh~ = the GPU's packed half-precision tanh approximation (absolute error
@@ -100,14 +120,15 @@ int sim_set_action_stream(sim_t *s, int mode);
  *       z2 = b2 + sum_k f16(W2[j][k]) * h1[k]   FP16 operands (b2 split in two parts), products exact,
  *                             fp32 accumulation in the order the tensor core chooses
  *       h2 = tanh~(f16(z2));  logits = b3 + W3 h2 with W3 and b3 split in two FP16 parts, fp32 accumulation.
- *     Parameters beyond the FP16 range (|x| > 65504) saturate.  Sampling, physics, reset and outputs are
- *     unchanged, so a trajectory stays an exact CartPole trajectory under the actions it records; only the
- *     action probabilities differ from exact mode, by the logit error, which is bounded by
+ *     The logit error is bounded by
  *       sum_j |W3[i][j]| (e + sum_k |W2[j][k]| (e + 2^-11 |h1[k]|)),  e = 2^-10.987 + 0.448 * 2^-11,
- *     and is far smaller for typical weights.  Not bit-reproducible across GPU generations.
- * The first call that selects tensor mode allocates a 4-byte device status word (see
+ *     and is far smaller for typical weights.
+ * In both tensor modes parameters beyond the FP16 range (|x| > 65504) saturate; sampling, physics, reset and
+ * outputs are unchanged, so a trajectory stays an exact CartPole trajectory under the actions it records; only the
+ * action probabilities differ from exact mode, by the logit error.  Not bit-reproducible across GPU generations.
+ * The first call that selects a tensor mode allocates a 4-byte device status word (see
  * sim_get_device_status). */
-enum { SIM_POLICY_EXACT = 0, SIM_POLICY_TENSOR = 1 };
+enum { SIM_POLICY_EXACT = 0, SIM_POLICY_TENSOR = 1, SIM_POLICY_TENSOR_PRECISE = 2 };
 int sim_set_policy_mode(sim_t *s, int mode);
 
 /* sim_get_device_status -- flags raised by kernels of this handle since it was created; synchronises the
@@ -125,7 +146,8 @@ int sim_get_device_status(sim_t *s, uint32_t *h_flags);
  * Uses a status word of its own: the handle's status (sim_get_device_status) is not touched. */
 int sim_selfcheck_tensor_wait(sim_t *s, uint32_t *h_status, uint32_t *h_threads_completed);
 
-/* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env. */
+/* sim_reset -- t = 0, ep_len = 0, reset_count = 0, state = draw #0 for every env: the initial state that the
+ * step() transition of Section 3.2 starts from. */
 int sim_reset(sim_t *s);
 
 /*
@@ -140,8 +162,8 @@ int sim_step(sim_t *s, const int8_t *d_actions, float *d_next_obs, float *d_rew,
 
 /*
  * sim_rollout -- T steps of every env in ceil(T / K_fused) kernel launches; inside one
- * launch the state lives in registers / shared memory (Section 4, "K simulator steps are
- * executed in a single fused GPU kernel launch").  K_fused = 1 is plain GPU vectorization.
+ * launch the state lives in registers / shared memory (Section 4: simulator kernel fusion runs
+ * K simulator steps in one kernel launch).  K_fused = 1 is plain GPU vectorization (Section 3).
  *   T >= 1, K_fused >= 1 (values above T are clamped to T).
  *   d_policy_params  NULL = uniform random actions; else SIM_POLICY_PARAM_COUNT floats of
  *                    the 4-64-64-2 tanh MLP whose softmax is sampled with the action word
@@ -168,13 +190,16 @@ int sim_rollout_host(sim_t *s, int T, int K_fused, const float *h_policy_params,
                      float *h_obs, int8_t *h_act, float *h_rew, uint8_t *h_done);
 
 /* Inspection and checkpoint hooks: copy state / counters out of or into the handle
- * (device pointers; d_* may be NULL to skip one).  h_t is a host pointer. */
+ * (device pointers; d_* may be NULL to skip one).  h_t is a host pointer.  (No passage of the paper:
+ * together with t and the seed these are the complete state of a rollout, so saving and restoring them
+ * resumes it exactly.) */
 int sim_get_state(sim_t *s, float *d_state /* [N,S] */);
 int sim_set_state(sim_t *s, const float *d_state /* [N,S] */);
 int sim_get_counters(sim_t *s, uint32_t *d_ep_len, uint32_t *d_reset_count, uint64_t *h_t);
 int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t *d_reset_count, uint64_t t);
 
-/* sim_policy_logits -- logits of the MLP for M observations (no sampling, no stepping).
+/* sim_policy_logits -- logits of the MLP for M observations (no sampling, no stepping): the inference half of
+ * the data-collection loop of Section 2.1 on its own, as a test and inspection hook.
  *   d_obs [M,4] fp32, d_params SIM_POLICY_PARAM_COUNT fp32, d_logits [M,2] fp32.  s may be
  *   any live handle (it provides the stream and the policy mode). */
 int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits);
@@ -187,8 +212,7 @@ int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_pa
 int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, float *d_obs6);
 
 /* sim_episode_returns -- running return of every episode of a trajectory, for consumers that label the
- * collected samples with returns (the paper: "reward is used to form labels for the collected data",
- * Section 2.1).  d_rew [T,n] fp32 and d_done [T,n] u8 as written by sim_rollout; d_ret [T,n] fp32 receives
+ * collected samples with returns (Section 2.1: the rewards become the labels of the collected data).  d_rew [T,n] fp32 and d_done [T,n] u8 as written by sim_rollout; d_ret [T,n] fp32 receives
  * ret[t,e] = rew[t,e] + (done[t-1,e] ? 0 : ret[t-1,e]), added in time order in fp32.  d_carry [n] fp32
  * (nullable) carries the return accumulated so far across calls: read before row 0, written after the last
  * row (0 where the episode just ended).  All device pointers. */
@@ -224,11 +248,17 @@ int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_mismatches);
  *   cuda_stream                         cudaStream_t as void*, NULL = default stream.  Work is
  *                                       only enqueued; the caller synchronises.
  * Limit: 256-aligned(4*state_dim*n_envs) + 2 * 256-aligned(4*n_envs) bytes must not exceed
- * SIM_NOALLOC_SCRATCH_BYTES (e.g. 349 440 four-float envs); larger problems return
+ * SIM_NOALLOC_SCRATCH_BYTES (at most 349 504 four-float envs); larger problems return
  * SIM_ECAPACITY and enqueue nothing.  Other errors: SIM_EINVAL, SIM_ECUDA.
  * The call makes no cudaMalloc, cudaFree or other allocating call, on the host or the device.
  * First use on a device looks up the array's device address (once per device, with that device
- * current): make that first call outside any stream capture.
+ * current): make that first call outside any stream capture.  With CUDA's lazy module loading that
+ * first lookup is also the moment the driver loads the library's device image, array included, and
+ * reserves its 8 MiB, which can fail if the device is full: callers that must not allocate later
+ * should make one small warm-up call at start-up.  From the second call on a device nothing is
+ * allocated by anyone (the test suite checks the device's free memory across such calls).
+ * The launches are planned exactly as in sim_rollout (same kernels for the same env kind, policy and
+ * launch length); the policy is evaluated in exact mode.
  * All calls share the one array.  It keeps the previous call's contents; each call rewrites every
  * word it later reads before reading it, so nothing needs clearing by the caller -- but two
  * calls whose work overlaps on the GPU (different streams, or one process-wide device shared by
@@ -239,11 +269,12 @@ int sim_rollout_noalloc(int env_kind, int64_t n_envs, int state_dim, uint64_t se
                         const float *d_policy_params, float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done,
                         void *cuda_stream);
 
-/* sim_launch_count -- kernels launched by this handle since creation (for launch accounting). */
+/* sim_launch_count -- kernels launched by this handle since creation (the launch accounting of Section 3.3:
+ * one launch per K_fused steps). */
 int64_t sim_launch_count(sim_t *s);
 
 /* sim_strerror -- static string for a SIM_* code.  sim_last_cuda_error -- the cudaError_t
- * behind the most recent SIM_ECUDA of this handle (0 if none). */
+ * behind the most recent SIM_ECUDA of this handle (0 if none).  (No passage of the paper: error reporting.) */
 const char *sim_strerror(int code);
 int sim_last_cuda_error(sim_t *s);
 

@@ -73,16 +73,6 @@ def lib() -> C.CDLL:
         L.oracle_mlp_logits.restype = None
         L.oracle_sample_action.argtypes = [f32p, C.c_uint32]
         L.oracle_sample_action.restype = C.c_int
-        L.oracle_rollout.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int64, C.c_void_p,
-                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_int,
-                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
-                                     C.c_void_p, C.c_void_p]
-        L.oracle_rollout.restype = C.c_int
-        L.oracle_rollout_c.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_int64, C.c_void_p,
-                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_int,
-                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
-                                       C.c_void_p, C.c_void_p]
-        L.oracle_rollout_c.restype = C.c_int
         L.oracle_rollout_x.argtypes = [C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_int, C.c_int64, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_int,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,

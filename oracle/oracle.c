@@ -491,32 +491,6 @@ ORACLE_API int oracle_rollout_x(int env_kind, int S, uint64_t seed, int compute_
     return 0;
 }
 
-/* Word-per-step action stream (the default). */
-ORACLE_API int oracle_rollout_c(int env_kind, int S, uint64_t seed, int compute_factor,
-                                int64_t n_sel, const uint32_t *env_ids,
-                                float *state, uint32_t *ep_len, uint32_t *reset_count,
-                                uint64_t t0, int T,
-                                const float *policy_params, const int8_t *given_actions,
-                                float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done,
-                                float *next_obs)
-{
-    return oracle_rollout_x(env_kind, S, seed, compute_factor, 0, n_sel, env_ids, state, ep_len, reset_count, t0, T,
-                            policy_params, given_actions, out_obs, out_act, out_rew, out_done, next_obs);
-}
-
-/* The plain simulator: compute factor 1. */
-ORACLE_API int oracle_rollout(int env_kind, int S, uint64_t seed,
-                              int64_t n_sel, const uint32_t *env_ids,
-                              float *state, uint32_t *ep_len, uint32_t *reset_count,
-                              uint64_t t0, int T,
-                              const float *policy_params, const int8_t *given_actions,
-                              float *out_obs, int8_t *out_act, float *out_rew, uint8_t *out_done,
-                              float *next_obs)
-{
-    return oracle_rollout_c(env_kind, S, seed, 1, n_sel, env_ids, state, ep_len, reset_count, t0, T,
-                            policy_params, given_actions, out_obs, out_act, out_rew, out_done, next_obs);
-}
-
 /* Running return of every episode in a trajectory: ret[t,e] = rew[t,e] + (done[t-1,e] ? 0 : ret[t-1,e]),
  * with `carry` [n] (in: return accumulated before row 0; out: after the last row, 0 where it ended). */
 ORACLE_API void oracle_episode_returns(const float *rew, const uint8_t *done, int T, int64_t n, float *carry, float *ret)

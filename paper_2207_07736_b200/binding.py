@@ -119,7 +119,7 @@ def sim_set_action_stream(h, mode):
     _check(lib().sim_set_action_stream(h, mode), h)
 
 
-SIM_POLICY_EXACT, SIM_POLICY_TENSOR = 0, 1
+SIM_POLICY_EXACT, SIM_POLICY_TENSOR, SIM_POLICY_TENSOR_PRECISE = 0, 1, 2
 SIM_STATUS_TENSOR_WAIT = 1
 
 

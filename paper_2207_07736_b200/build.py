@@ -10,7 +10,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libsim_b200.so"
-SOURCES = ["sim_api.cu", "sim_noalloc.cu", "rollout_s4.cu", "rollout_cartpole.cu", "rollout_acrobot.cu", "rollout_mlp.cu", "rollout_mlp_tc.cu", "rollout_synth.cu"]
+SOURCES = ["sim_api.cu", "sim_noalloc.cu", "rollout_s4.cu", "rollout_cartpole.cu", "rollout_acrobot.cu", "rollout_mlp.cu", "rollout_mlp_tc.cu", "rollout_mlp_tcp.cu", "rollout_synth.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--fmad=false", "-prec-div=true", "-prec-sqrt=true", "-ftz=false",

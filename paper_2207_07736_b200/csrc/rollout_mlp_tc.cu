@@ -24,14 +24,16 @@
 // the first 4 KB of the tile's A2 buffer (it is dead before h1 is written).
 // Every wait is bounded: when a barrier does not complete in time the group records bit 0 in the status
 // word and skips its remaining steps; the CTA then frees its TMEM columns and returns.
+#include <mutex>
+
 #include "sim_internal.h"
 #include "sim_envs.cuh"
+#include "tc_common.cuh"
 
 namespace simk {
 
 constexpr int kTcThreads = 256;                   // per CTA
 constexpr uint32_t kTile = 128u;                  // envs (rows) per tile = threads per group
-constexpr uint32_t kTcLBO = 128u;                 // bytes between core matrices adjacent along K
 constexpr uint32_t kCh1 = 2u, kCh2 = 10u;         // 16-byte chunks per operand row: 16 and 80 FP16 values
 constexpr uint32_t kTileCols = 64u;               // TMEM columns (fp32) per tile: z1 / z2 use all, the logits the first 16
 constexpr uint32_t kTcCols = 2u * kTileCols;
@@ -56,30 +58,6 @@ struct TcCtx {
     uint32_t row;           // thread index inside the group
     bool fail;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// f16x2 with `first` in the low half (the lower address / lower k).
-__device__ __forceinline__ uint32_t pack_f16x2(float first, float second) { uint32_t r; asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(second), "f"(first)); return r; }
-__device__ __forceinline__ uint32_t tanh_f16x2(uint32_t x) { uint32_t r; asm("tanh.approx.f16x2 %0, %1;" : "=r"(r) : "r"(x)); return r; }
-__device__ __forceinline__ uint16_t f16_bits(float x) { uint16_t r; asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(r) : "f"(x)); return r; }
-__device__ __forceinline__ float f16_value(uint16_t h) { float r; asm("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(h)); return r; }
-// x = hi + lo with hi = f16(x), lo = f16(x - hi).
-__device__ __forceinline__ void f16_split(float x, uint16_t &hi, uint16_t &lo) { hi = f16_bits(x); lo = f16_bits(__fsub_rn(x, f16_value(hi))); }
-
-// Shared-memory matrix descriptor: start address, leading and stride byte offsets (16-byte units),
-// descriptor version 1, no swizzle.
-__device__ __forceinline__ uint64_t tc_desc(uint32_t saddr, uint32_t chunks_per_row)
-{
-    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)(kTcLBO >> 4) << 16) | ((uint64_t)((chunks_per_row * 128u) >> 4) << 32) | (1ull << 46);
-}
-
-// Index (in 16-byte chunks) of chunk c of row `row` of an operand tile with `ch` chunks per row.
-__device__ __forceinline__ uint32_t tc_chunk(uint32_t row, uint32_t c, uint32_t ch) { return (row >> 3) * ch * 8u + c * 8u + (row & 7u); }
-
-__device__ __forceinline__ void tc_put(uint4 *tile, uint32_t row, uint32_t k, uint32_t ch, uint16_t value)
-{
-    reinterpret_cast<uint16_t *>(tile + tc_chunk(row, k >> 3, ch))[k & 7u] = value;
-}
 
 // Group barrier (named barrier 1 + group, 128 threads) with an OR reduction of `flag`.
 __device__ __forceinline__ bool group_sync_or(uint32_t group, bool flag)
@@ -185,29 +163,11 @@ __device__ __forceinline__ bool tc_contract(TcSmem &s, TcCtx &c, uint32_t *statu
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
     }
-    uint32_t done = 0u;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(bar), "r"(c.parity) : "memory");
-    if (!done) {                                                       // rare: the first wait timed out inside the hardware
-        const long long t0 = clock64();
-        do {
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                         : "=r"(done) : "r"(bar), "r"(c.parity) : "memory");
-        } while (!done && clock64() - t0 <= wait_cycles);
-    }
+    const bool done = mbarrier_wait_bounded(bar, c.parity, wait_cycles);
     if (!done) { c.fail = true; if (status) atomicOr(status, 1u); }
     c.parity ^= 1u;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     return true;
-}
-
-// Columns 0..15 from `taddr` of this thread's accumulator row.
-__device__ __forceinline__ void tc_load16(uint32_t taddr, uint32_t (&v)[16])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-                 : "r"(taddr));
 }
 
 // My accumulator row (64 columns) -> tanh -> FP16 -> my row of the group's A2 operand.
@@ -348,10 +308,12 @@ tensor_wait_selfcheck_kernel(const float *__restrict__ params, long long wait_cy
 // The kernels need more than 48 KB of dynamic shared memory: opt in once per device.
 static cudaError_t tc_opt_in()
 {
+    static std::mutex lock;
     static bool done[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> guard(lock);
     if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
     e = cudaFuncSetAttribute(rollout_cartpole_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(policy_logits_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TcSmem));

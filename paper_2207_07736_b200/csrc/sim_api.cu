@@ -11,23 +11,10 @@
 
 using namespace simk;
 
-struct sim {
-    int env_kind;
-    int S;
-    uint32_t n;
+struct sim : SimCore {           // the population (kind, sizes, buffers, keys, t) is the part the launch planner sees
     uint64_t seed;
-    uint64_t env_offset;
-    uint64_t t;
-    int compute_factor;
-    int action_stream;
-    int policy_mode;
-    uint32_t *d_status;       // device status word, allocated when tensor mode is first selected
-    int device;
+    int device;               // ordinal of the device the handle was created on; every call must find it current
     cudaStream_t stream;
-    float *state;
-    uint32_t *ep_len;
-    uint32_t *reset_count;
-    RoundKeys rk;
     int last_cuda;
     int64_t launches;
     // staging for sim_rollout_host (allocated on first use)
@@ -47,7 +34,7 @@ static int cuda_fail(sim *s, cudaError_t e)
 }
 #define CU(s, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((s), e_); } while (0)
 
-static void expand_keys(uint64_t seed, RoundKeys &rk)
+void simk::expand_round_keys(uint64_t seed, RoundKeys &rk)
 {
     uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFu), k1 = (uint32_t)(seed >> 32);
     for (int r = 0; r < 10; ++r) {
@@ -55,6 +42,17 @@ static void expand_keys(uint64_t seed, RoundKeys &rk)
         k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
     }
 }
+
+// A handle's buffers live on the device it was created on: a call made with another device current would
+// launch there on pointers that device cannot use.  Host check only.
+static int check_device(sim *s)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(s, e);
+    return dev == s->device ? SIM_OK : SIM_ESTATE;
+}
+#define DEV(s) do { int rc_ = check_device(s); if (rc_ != SIM_OK) return rc_; } while (0)
 
 static bool valid_state_dim(int env_kind, int S)
 {
@@ -69,7 +67,7 @@ SIM_API const char *sim_strerror(int code)
     case SIM_EINVAL: return "invalid argument";
     case SIM_ENOMEM: return "out of device memory";
     case SIM_ECUDA: return "CUDA error (see sim_last_cuda_error)";
-    case SIM_ESTATE: return "call not valid in the handle's current state";
+    case SIM_ESTATE: return "call not valid in the handle's current state (e.g. another CUDA device is current than the one it was created on)";
     case SIM_ECAPACITY: return "problem does not fit the fixed scratch array of the no-allocation entry point";
     default: return "unknown error code";
     }
@@ -103,12 +101,11 @@ SIM_API int sim_create(sim_t **out, int env_kind, int64_t n_envs, int state_dim,
     if (n_envs < 1 || n_envs > 0xFFFFFFFFll) return SIM_EINVAL;
     if (!valid_state_dim(env_kind, state_dim)) return SIM_EINVAL;
 
-    sim *s = new (std::nothrow) sim();
+    sim *s = new (std::nothrow) sim();          // value-initialised: every field starts at zero
     if (!s) return SIM_ENOMEM;
-    memset(s, 0, sizeof(*s));
     s->env_kind = env_kind; s->S = state_dim; s->n = (uint32_t)n_envs; s->seed = seed;
     s->compute_factor = 1;
-    expand_keys(seed, s->rk);
+    expand_round_keys(seed, s->rk);
     cudaError_t e = cudaGetDevice(&s->device);
     if (e == cudaSuccess) e = cudaMalloc(&s->state, (size_t)n_envs * (size_t)state_dim * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&s->ep_len, (size_t)n_envs * sizeof(uint32_t));
@@ -165,9 +162,10 @@ SIM_API int sim_set_action_stream(sim_t *s, int mode)
 
 SIM_API int sim_set_policy_mode(sim_t *s, int mode)
 {
-    if (!s || (mode != SIM_POLICY_EXACT && mode != SIM_POLICY_TENSOR)) return SIM_EINVAL;
-    if (mode == SIM_POLICY_TENSOR && s->env_kind != SIM_CARTPOLE) return SIM_EINVAL;
-    if (mode == SIM_POLICY_TENSOR && !s->d_status) {
+    if (!s || (mode != SIM_POLICY_EXACT && mode != SIM_POLICY_TENSOR && mode != SIM_POLICY_TENSOR_PRECISE)) return SIM_EINVAL;
+    if (mode != SIM_POLICY_EXACT && s->env_kind != SIM_CARTPOLE) return SIM_EINVAL;
+    if (mode != SIM_POLICY_EXACT && !s->d_status) {
+        DEV(s);
         CU(s, cudaMalloc(&s->d_status, sizeof(uint32_t)));
         CU(s, cudaMemsetAsync(s->d_status, 0, sizeof(uint32_t), s->stream));
     }
@@ -180,6 +178,7 @@ SIM_API int sim_get_device_status(sim_t *s, uint32_t *h_flags)
     if (!s || !h_flags) return SIM_EINVAL;
     *h_flags = 0u;
     if (!s->d_status) return SIM_OK;
+    DEV(s);
     CU(s, cudaMemcpyAsync(h_flags, s->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s->stream));
     CU(s, cudaStreamSynchronize(s->stream));
     return SIM_OK;
@@ -188,43 +187,51 @@ SIM_API int sim_get_device_status(sim_t *s, uint32_t *h_flags)
 SIM_API int sim_reset(sim_t *s)
 {
     if (!s) return SIM_EINVAL;
+    DEV(s);
     CU(s, launch_reset(s->env_kind, s->S, s->state, s->ep_len, s->reset_count, s->n, (uint32_t)s->env_offset, s->rk, s->stream));
     s->launches += 1;
     s->t = 0;
     return SIM_OK;
 }
 
-// One launch of K steps starting at the handle's current t.  Output pointers address row 0 of this launch.
+// One launch of K steps of the population `c`, starting at c.t: picks the kernel for the env kind, the policy and
+// the launch length.  Output pointers address row 0 of this launch.  Shared by every entry point that rolls out.
+cudaError_t simk::launch_planned(const SimCore &c, int K, int policy, const float *d_params, const int8_t *d_actions, float *next_obs,
+                                 float *obs, int8_t *act, float *rew, uint8_t *done, cudaStream_t st)
+{
+    const uint32_t tb0 = (uint32_t)(c.t >> 2);
+    const int phase = (int)(c.t & 3);
+    if (c.env_kind == SIM_SYNTH) {
+        SynthArgs a;
+        a.state = c.state; a.ep_len = c.ep_len; a.reset_count = c.reset_count;
+        a.n = c.n; a.env_offset = (uint32_t)c.env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = c.compute_factor;
+        a.out_obs = obs; a.out_act = act; a.out_rew = rew; a.out_done = done;
+        a.actions = d_actions; a.next_obs = next_obs; a.rk = c.rk;
+        return launch_synth(c.S, a, st);
+    }
+    S4Args a;
+    a.state = reinterpret_cast<float4 *>(c.state); a.ep_len = c.ep_len; a.reset_count = c.reset_count;
+    a.n = c.n; a.env_offset = (uint32_t)c.env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = c.compute_factor;
+    a.out_obs = reinterpret_cast<float4 *>(obs); a.out_act = act; a.out_rew = rew; a.out_done = done;
+    a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.status = c.d_status; a.rk = c.rk;
+    a.action_bits = (c.action_stream == SIM_ACTIONS_BITS && policy == POLICY_RANDOM) ? 1 : 0;
+    if (c.env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM && c.compute_factor == 1)
+        return launch_cartpole_random(a, st);
+    if (c.env_kind == SIM_ACROBOT && policy == POLICY_RANDOM && K > 4)      // short launches: the scalar kernel has the shorter step latency
+        return launch_acrobot_random(a, st);
+    if (c.env_kind == SIM_CARTPOLE && policy == POLICY_MLP && c.policy_mode == SIM_POLICY_TENSOR)
+        return launch_cartpole_mlp_tc(a, st);
+    if (c.env_kind == SIM_CARTPOLE && policy == POLICY_MLP && c.policy_mode == SIM_POLICY_TENSOR_PRECISE)
+        return launch_cartpole_mlp_tcp(a, st);
+    if (c.env_kind == SIM_CARTPOLE && policy == POLICY_MLP)
+        return launch_cartpole_mlp(a, st);
+    return launch_s4(c.env_kind, policy, a, st);
+}
+
 static int launch_chunk(sim *s, int K, int policy, const float *d_params, const int8_t *d_actions, float *next_obs,
                         float *obs, int8_t *act, float *rew, uint8_t *done)
 {
-    const uint32_t tb0 = (uint32_t)(s->t >> 2);
-    const int phase = (int)(s->t & 3);
-    if (s->env_kind == SIM_SYNTH) {
-        SynthArgs a;
-        a.state = s->state; a.ep_len = s->ep_len; a.reset_count = s->reset_count;
-        a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = s->compute_factor;
-        a.out_obs = obs; a.out_act = act; a.out_rew = rew; a.out_done = done;
-        a.actions = d_actions; a.next_obs = next_obs; a.rk = s->rk;
-        CU(s, launch_synth(s->S, a, s->stream));
-    } else {
-        S4Args a;
-        a.state = reinterpret_cast<float4 *>(s->state); a.ep_len = s->ep_len; a.reset_count = s->reset_count;
-        a.n = s->n; a.env_offset = (uint32_t)s->env_offset; a.tb0 = tb0; a.phase = phase; a.K = K; a.C = s->compute_factor;
-        a.out_obs = reinterpret_cast<float4 *>(obs); a.out_act = act; a.out_rew = rew; a.out_done = done;
-        a.actions = d_actions; a.next_obs = reinterpret_cast<float4 *>(next_obs); a.params = d_params; a.status = s->d_status; a.rk = s->rk;
-        a.action_bits = (s->action_stream == SIM_ACTIONS_BITS && policy == POLICY_RANDOM) ? 1 : 0;
-        if (s->env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM && s->compute_factor == 1)
-            CU(s, launch_cartpole_random(a, s->stream));
-        else if (s->env_kind == SIM_ACROBOT && policy == POLICY_RANDOM && K > 4)      // short launches: the scalar kernel has the shorter step latency
-            CU(s, launch_acrobot_random(a, s->stream));
-        else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP && s->policy_mode == SIM_POLICY_TENSOR)
-            CU(s, launch_cartpole_mlp_tc(a, s->stream));
-        else if (s->env_kind == SIM_CARTPOLE && policy == POLICY_MLP)
-            CU(s, launch_cartpole_mlp(a, s->stream));
-        else
-            CU(s, launch_s4(s->env_kind, policy, a, s->stream));
-    }
+    CU(s, launch_planned(*s, K, policy, d_params, d_actions, next_obs, obs, act, rew, done, s->stream));
     s->launches += 1;
     s->t += (uint64_t)K;
     return SIM_OK;
@@ -233,6 +240,7 @@ static int launch_chunk(sim *s, int K, int policy, const float *d_params, const 
 SIM_API int sim_step(sim_t *s, const int8_t *d_actions, float *d_next_obs, float *d_rew, uint8_t *d_done)
 {
     if (!s || !d_actions) return SIM_EINVAL;
+    DEV(s);
     return launch_chunk(s, 1, POLICY_GIVEN, nullptr, d_actions, d_next_obs, nullptr, nullptr, d_rew, d_done);
 }
 
@@ -248,6 +256,7 @@ SIM_API int sim_rollout(sim_t *s, int T, int K_fused, const float *d_policy_para
 {
     int rc = check_rollout_args(s, T, K_fused, d_policy_params);
     if (rc != SIM_OK) return rc;
+    DEV(s);
     const int K = K_fused > T ? T : K_fused;
     const int policy = d_policy_params ? POLICY_MLP : POLICY_RANDOM;
     const size_t n = s->n, S = (size_t)s->S;
@@ -273,6 +282,7 @@ SIM_API int sim_rollout_host(sim_t *s, int T, int K_fused, const float *h_policy
 {
     int rc = check_rollout_args(s, T, K_fused, h_policy_params);
     if (rc != SIM_OK) return rc;
+    DEV(s);
     const int K = K_fused > T ? T : K_fused;
     const size_t n = s->n, S = (size_t)s->S;
     const size_t rows = (size_t)K * n;
@@ -334,6 +344,7 @@ SIM_API int sim_rollout_host(sim_t *s, int T, int K_fused, const float *h_policy
 SIM_API int sim_get_state(sim_t *s, float *d_state)
 {
     if (!s || !d_state) return SIM_EINVAL;
+    DEV(s);
     CU(s, cudaMemcpyAsync(d_state, s->state, (size_t)s->n * s->S * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
     return SIM_OK;
 }
@@ -341,6 +352,7 @@ SIM_API int sim_get_state(sim_t *s, float *d_state)
 SIM_API int sim_set_state(sim_t *s, const float *d_state)
 {
     if (!s || !d_state) return SIM_EINVAL;
+    DEV(s);
     CU(s, cudaMemcpyAsync(s->state, d_state, (size_t)s->n * s->S * sizeof(float), cudaMemcpyDeviceToDevice, s->stream));
     return SIM_OK;
 }
@@ -348,6 +360,7 @@ SIM_API int sim_set_state(sim_t *s, const float *d_state)
 SIM_API int sim_get_counters(sim_t *s, uint32_t *d_ep_len, uint32_t *d_reset_count, uint64_t *h_t)
 {
     if (!s) return SIM_EINVAL;
+    DEV(s);
     if (d_ep_len) CU(s, cudaMemcpyAsync(d_ep_len, s->ep_len, (size_t)s->n * 4, cudaMemcpyDeviceToDevice, s->stream));
     if (d_reset_count) CU(s, cudaMemcpyAsync(d_reset_count, s->reset_count, (size_t)s->n * 4, cudaMemcpyDeviceToDevice, s->stream));
     if (h_t) *h_t = s->t;
@@ -357,6 +370,7 @@ SIM_API int sim_get_counters(sim_t *s, uint32_t *d_ep_len, uint32_t *d_reset_cou
 SIM_API int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t *d_reset_count, uint64_t t)
 {
     if (!s) return SIM_EINVAL;
+    DEV(s);
     if (d_ep_len) CU(s, cudaMemcpyAsync(s->ep_len, d_ep_len, (size_t)s->n * 4, cudaMemcpyDeviceToDevice, s->stream));
     if (d_reset_count) CU(s, cudaMemcpyAsync(s->reset_count, d_reset_count, (size_t)s->n * 4, cudaMemcpyDeviceToDevice, s->stream));
     s->t = t;
@@ -366,8 +380,11 @@ SIM_API int sim_set_counters(sim_t *s, const uint32_t *d_ep_len, const uint32_t 
 SIM_API int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const float *d_params, float *d_logits)
 {
     if (!s || !d_obs || !d_params || !d_logits || M < 0) return SIM_EINVAL;
+    DEV(s);
     if (s->policy_mode == SIM_POLICY_TENSOR)
         CU(s, launch_policy_logits_tc(d_obs, M, d_params, d_logits, s->d_status, s->stream));
+    else if (s->policy_mode == SIM_POLICY_TENSOR_PRECISE)
+        CU(s, launch_policy_logits_tcp(d_obs, M, d_params, d_logits, s->d_status, s->stream));
     else
         CU(s, launch_policy_logits(d_obs, M, d_params, d_logits, s->stream));
     if (M > 0) s->launches += 1;
@@ -377,6 +394,7 @@ SIM_API int sim_policy_logits(sim_t *s, const float *d_obs, int64_t M, const flo
 SIM_API int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_mismatches)
 {
     if (!s || !h_mismatches || nums_per_den < 0) return SIM_EINVAL;
+    DEV(s);
     unsigned long long *d_bad = nullptr;
     CU(s, cudaMalloc(&d_bad, sizeof(unsigned long long)));
     cudaError_t e = cudaMemsetAsync(d_bad, 0, sizeof(unsigned long long), s->stream);
@@ -396,6 +414,7 @@ SIM_API int sim_selfcheck_division(sim_t *s, int nums_per_den, uint64_t *h_misma
 SIM_API int sim_selfcheck_tensor_wait(sim_t *s, uint32_t *h_status, uint32_t *h_threads_completed)
 {
     if (!s || !h_status || !h_threads_completed) return SIM_EINVAL;
+    DEV(s);
     const size_t words = SIM_POLICY_PARAM_COUNT + 1 + 256;
     uint32_t *d = nullptr;
     CU(s, cudaMalloc(&d, words * sizeof(uint32_t)));
@@ -417,6 +436,7 @@ SIM_API int sim_selfcheck_tensor_wait(sim_t *s, uint32_t *h_status, uint32_t *h_
 SIM_API int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, float *d_obs6)
 {
     if (!s || !d_state || !d_obs6 || M < 0) return SIM_EINVAL;
+    DEV(s);
     CU(s, launch_acrobot_observation(d_state, M, d_obs6, s->stream));
     if (M > 0) s->launches += 1;
     return SIM_OK;
@@ -425,6 +445,7 @@ SIM_API int sim_acrobot_observation(sim_t *s, const float *d_state, int64_t M, f
 SIM_API int sim_episode_returns(sim_t *s, const float *d_rew, const uint8_t *d_done, int T, int64_t n, float *d_carry, float *d_ret)
 {
     if (!s || !d_rew || !d_done || !d_ret || T < 0 || n < 0) return SIM_EINVAL;
+    DEV(s);
     CU(s, launch_episode_returns(d_rew, d_done, T, n, d_carry, d_ret, s->stream));
     if (T > 0 && n > 0) s->launches += 1;
     return SIM_OK;

@@ -52,6 +52,24 @@ struct SynthArgs {
     RoundKeys rk;
 };
 
+// One population of envs as the launch planner sees it: kind, sizes, where its buffers live, keys, the step counter
+// and the per-handle options.  A handle of the C ABI is one of these plus host-side bookkeeping.
+struct SimCore {
+    int env_kind;
+    int S;
+    uint32_t n;
+    uint64_t env_offset;
+    uint64_t t;               // global step index of the next step
+    int compute_factor;
+    int action_stream;
+    int policy_mode;
+    uint32_t *d_status;       // device status word (tensor policy modes), nullable
+    float *state;             // [n, S]
+    uint32_t *ep_len;         // [n]
+    uint32_t *reset_count;    // [n]
+    RoundKeys rk;
+};
+
 // Programmatic dependent launch: consecutive rollout launches of one stream overlap their launch
 // latency.  A kernel calls pdl_wait() before its first global-memory access (it returns once every
 // earlier grid of the stream has completed and its writes are visible; a no-op when the launch did not
@@ -77,6 +95,11 @@ static inline cudaError_t launch_overlapped(bool overlap, void (*kernel)(KArgs..
 }
 #endif
 
+void expand_round_keys(uint64_t seed, RoundKeys &rk);
+// The launch planner: one launch of K steps of population `c` from step c.t (it advances nothing itself).
+cudaError_t launch_planned(const SimCore &c, int K, int policy, const float *d_params, const int8_t *d_actions, float *next_obs,
+                           float *obs, int8_t *act, float *rew, uint8_t *done, cudaStream_t st);
+
 // Launchers (each returns the launch error, enqueues on `st`, never synchronises).
 cudaError_t launch_reset(int env_kind, int S, float *state, uint32_t *ep_len, uint32_t *reset_count,
                          uint32_t n, uint32_t env_offset, const RoundKeys &rk, cudaStream_t st);
@@ -85,6 +108,8 @@ cudaError_t launch_cartpole_random(const S4Args &a, cudaStream_t st);   // CartP
 cudaError_t launch_acrobot_random(const S4Args &a, cudaStream_t st);    // Acrobot, uniform random torque, packed two-env kernel
 cudaError_t launch_cartpole_mlp(const S4Args &a, cudaStream_t st);      // CartPole, MLP policy, packed two-env kernel
 cudaError_t launch_cartpole_mlp_tc(const S4Args &a, cudaStream_t st);   // CartPole, MLP policy in tensor mode (tcgen05 hidden layer)
+cudaError_t launch_cartpole_mlp_tcp(const S4Args &a, cudaStream_t st);  // the same with split operands and fp32 tanh (precise tensor mode)
+cudaError_t launch_policy_logits_tcp(const float *obs, int64_t M, const float *params, float *logits, uint32_t *status, cudaStream_t st);
 cudaError_t launch_policy_logits_tc(const float *obs, int64_t M, const float *params, float *logits, uint32_t *status, cudaStream_t st);
 cudaError_t launch_tensor_wait_selfcheck(const float *params, long long wait_cycles, uint32_t *status, uint32_t *completed, cudaStream_t st);   // 256 words
 cudaError_t launch_division_selfcheck(int nums_per_den, unsigned long long *d_bad, cudaStream_t st);

@@ -77,40 +77,26 @@ int sim_rollout_noalloc(int env_kind, int64_t n_envs, int state_dim, uint64_t se
     uint32_t *reset_count = reinterpret_cast<uint32_t *>(base + off_rc);
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
-    RoundKeys rk;
-    {
-        uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFu), k1 = (uint32_t)(seed >> 32);
-        for (int r = 0; r < 10; ++r) { rk.k[r][0] = k0; rk.k[r][1] = k1; k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
-    }
+    // The population lives in the fixed array; everything else is what a fresh handle would hold.
+    SimCore c = {};
+    c.env_kind = env_kind; c.S = state_dim; c.n = (uint32_t)n; c.env_offset = 0; c.t = 0;
+    c.compute_factor = 1; c.action_stream = SIM_ACTIONS_WORD; c.policy_mode = SIM_POLICY_EXACT; c.d_status = nullptr;
+    c.state = state; c.ep_len = ep_len; c.reset_count = reset_count;
+    expand_round_keys(seed, c.rk);
     // the array keeps whatever the previous call left: the reset kernel rewrites every word this call reads
-    if (launch_reset(env_kind, state_dim, state, ep_len, reset_count, (uint32_t)n, 0u, rk, st) != cudaSuccess) { cudaGetLastError(); return SIM_ECUDA; }
+    if (launch_reset(env_kind, state_dim, state, ep_len, reset_count, c.n, 0u, c.rk, st) != cudaSuccess) { cudaGetLastError(); return SIM_ECUDA; }
 
+    // the same launch planner as sim_rollout: the same kernels for the same (env kind, policy, launch length)
     const int K = K_fused > T ? T : K_fused;
     const int policy = d_policy_params ? POLICY_MLP : POLICY_RANDOM;
     for (int t = 0; t < T; t += K) {
         const int k = (T - t) < K ? (T - t) : K;
         const size_t r0 = (size_t)t * n;
-        cudaError_t e;
-        if (env_kind == SIM_SYNTH) {
-            SynthArgs a;
-            a.state = state; a.ep_len = ep_len; a.reset_count = reset_count; a.n = (uint32_t)n; a.env_offset = 0u;
-            a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k; a.C = 1;
-            a.out_obs = out_obs ? out_obs + r0 * S : nullptr; a.out_act = out_act ? out_act + r0 : nullptr;
-            a.out_rew = out_rew ? out_rew + r0 : nullptr; a.out_done = out_done ? out_done + r0 : nullptr;
-            a.actions = nullptr; a.next_obs = nullptr; a.rk = rk;
-            e = launch_synth(state_dim, a, st);
-        } else {
-            S4Args a;
-            a.state = reinterpret_cast<float4 *>(state); a.ep_len = ep_len; a.reset_count = reset_count; a.n = (uint32_t)n; a.env_offset = 0u;
-            a.tb0 = (uint32_t)(t >> 2); a.phase = t & 3; a.K = k; a.C = 1;
-            a.out_obs = out_obs ? reinterpret_cast<float4 *>(out_obs) + r0 : nullptr; a.out_act = out_act ? out_act + r0 : nullptr;
-            a.out_rew = out_rew ? out_rew + r0 : nullptr; a.out_done = out_done ? out_done + r0 : nullptr;
-            a.actions = nullptr; a.next_obs = nullptr; a.params = d_policy_params; a.status = nullptr; a.rk = rk; a.action_bits = 0;
-            if (env_kind == SIM_CARTPOLE && policy == POLICY_RANDOM) e = launch_cartpole_random(a, st);
-            else if (env_kind == SIM_CARTPOLE) e = launch_cartpole_mlp(a, st);
-            else e = launch_s4(env_kind, policy, a, st);
-        }
+        const cudaError_t e = launch_planned(c, k, policy, d_policy_params, nullptr, nullptr,
+                                             out_obs ? out_obs + r0 * S : nullptr, out_act ? out_act + r0 : nullptr,
+                                             out_rew ? out_rew + r0 : nullptr, out_done ? out_done + r0 : nullptr, st);
         if (e != cudaSuccess) { cudaGetLastError(); return SIM_ECUDA; }
+        c.t += (uint64_t)k;
     }
     return SIM_OK;
 }

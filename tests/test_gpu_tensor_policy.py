@@ -130,7 +130,7 @@ def test_tensor_mode_argument_errors():
     acro = binding.Sim(oracle.ACROBOT, 16)
     assert binding.lib().sim_set_policy_mode(acro.h, binding.SIM_POLICY_TENSOR) == binding.SIM_EINVAL
     cp = binding.Sim(oracle.CARTPOLE, 16)
-    assert binding.lib().sim_set_policy_mode(cp.h, 2) == binding.SIM_EINVAL
+    assert binding.lib().sim_set_policy_mode(cp.h, 3) == binding.SIM_EINVAL
     assert binding.lib().sim_set_policy_mode(None, 0) == binding.SIM_EINVAL
     assert cp.device_status() == 0              # never selected: no status word, reads as clean
 

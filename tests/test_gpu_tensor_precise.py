@@ -1,0 +1,204 @@
+"""Precise tensor-mode MLP policy (SIM_POLICY_TENSOR_PRECISE): the three layers run as FP16 tensor-core
+contractions whose operands are split into exact FP16 parts, tanh is evaluated in fp32.  The stated tolerance of
+the benchmark's tolerance mode applies:
+  * logits within 1e-5 (absolute) of the oracle's fp32 logits, on >= 1e5 observations, for the harness weights,
+    for weights with biases, and for hostile ones (scaled up until tanh saturates and the logits reach several units);
+  * a rollout is an exact CartPole trajectory under the actions it records (the oracle, stepping with those actions,
+    reproduces every observation, reward, done flag, the final state and the counters bit for bit);
+  * a recorded action may differ from the oracle's decision on the recorded observation only where the uniform
+    draw lies within the probability change the asserted logit error can cause (|u - p0| <= tol / 2 + rounding
+    slack): such env-steps are ambiguous.  Differing and ambiguous env-steps are counted; at the full cfg3 size
+    (harness weights, asserted logit error 3e-6) both must stay below 1e-5 of the env-steps.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2207_07736_b200 import binding, inputs
+from gpu_common import assert_same_bits, to_np, torch_cuda
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = 1e-5                                  # the stated tolerance, asserted for every weight set
+HARNESS_TOL = 3e-6                                # asserted in addition for the cfg3 harness weights (seed 1, no biases)
+
+
+def p0_margin(logit_tol):
+    """Largest change of p0 = softmax(l)[0] a logit error of `logit_tol` per logit can cause (|d p0| <= |d(l0 - l1)| / 4),
+    plus the fp32 rounding of the oracle's own comparison."""
+    return 0.25 * 2 * logit_tol + 2e-7
+
+
+def exact_logits(p, obs):
+    return np.stack([oracle.mlp_logits(p, o) for o in obs])
+
+
+def scaled_params(seed, bias, scale):
+    p = inputs.mlp_params(seed, bias).copy()
+    p[0:256] *= scale
+    p[320:4416] *= scale
+    p[4480:4608] *= scale
+    return p.astype(np.float32)
+
+
+@pytest.mark.parametrize("seed,bias,scale", [(1, 0.0, 1.0), (7, 0.3, 1.0), (5, 1.0, 2.0), (9, 0.5, 3.0)])
+def test_precise_logits_within_1e5(seed, bias, scale):
+    torch = torch_cuda()
+    rng = np.random.default_rng(seed)
+    M = 120_007                                                    # many CTAs and a ragged tail
+    obs = (rng.uniform(-1, 1, (M, 4)) * np.array([2.4, 3, 0.21, 3])).astype(np.float32)
+    obs[:64] = 0.0                                                 # rest state
+    obs[64:128] *= np.float32(4.0)                                 # far outside what an episode reaches
+    obs[128:192] *= np.float32(1e-4)                               # tiny values: the low parts of the split go subnormal
+    p = scaled_params(seed, bias, scale)
+    sim = binding.Sim(oracle.CARTPOLE, 8, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE)
+    got = to_np(sim.policy_logits(torch.from_numpy(obs).cuda(), torch.from_numpy(p).cuda())).astype(np.float64)
+    assert sim.device_status() == 0
+    want = exact_logits(p, obs).astype(np.float64)
+    err = np.abs(got - want)
+    assert err.max() <= LOGIT_TOL, (err.max(), np.unravel_index(err.argmax(), err.shape), np.abs(want).max())
+    assert np.sqrt((err ** 2).mean()) <= 2e-6
+    if (seed, bias, scale) == (1, 0.0, 1.0):
+        assert err.max() <= HARNESS_TOL, err.max()
+    assert np.abs(want).max() > (0.5 if scale == 1.0 else 3.0)      # the logits are not trivially small
+    print("precise logits: seed %d bias %.1f scale %.1f  max err %.3g  rms %.3g  max |logit| %.2f" % (
+        seed, bias, scale, err.max(), np.sqrt((err ** 2).mean()), np.abs(want).max()))
+
+
+def check_precise_rollout(view, g, p, seed, env_ids, T, what, logit_tol=LOGIT_TOL):
+    """g: dict of numpy arrays [T, len(env_ids), ...] recorded by the GPU for the envs `env_ids` (global indices);
+    view.state() / view.counters() give the handle's final state restricted to those envs.  Returns
+    (differing actions, env-steps whose draw lies inside the ambiguity margin, env-steps)."""
+    assert set(np.unique(g["act"]).tolist()) <= {0, 1}
+    # 1. exact physics under the recorded actions
+    orc = oracle.OracleSim(oracle.CARTPOLE, seed=seed, env_ids=env_ids)
+    ref = orc.rollout(T, actions=g["act"])
+    for k in ("obs", "rew", "done"):
+        assert_same_bits(g[k], ref[k], "%s %s under the recorded actions" % (what, k))
+    assert_same_bits(to_np(view.state()), orc.state, what + " final state")
+    ep, rc, t = view.counters()
+    assert_same_bits(to_np(ep).astype(np.uint32), orc.ep_len, what + " ep_len")
+    assert_same_bits(to_np(rc).astype(np.uint32), orc.reset_count, what + " reset_count")
+    assert t == T
+    # 2. recorded actions against the oracle's decision on the recorded observations
+    flat_obs = g["obs"].reshape(-1, 4)
+    lg = exact_logits(p, flat_obs)
+    p0 = 1.0 / (1.0 + np.exp(lg[:, 1].astype(np.float64) - lg[:, 0].astype(np.float64)))
+    differ = ambiguous = 0
+    n = len(env_ids)
+    margin = p0_margin(logit_tol)
+    for idx in range(flat_obs.shape[0]):
+        t_, c = divmod(idx, n)
+        w = oracle.action_word(seed, int(env_ids[c]), t_)
+        u = float(oracle.uniform01(w))
+        near = abs(u - p0[idx]) <= margin
+        ambiguous += int(near)
+        if int(g["act"][t_, c]) != oracle.sample_action(lg[idx], w):
+            differ += 1
+            assert near, (what, t_, c, u, p0[idx])
+    return differ, ambiguous, flat_obs.shape[0]
+
+
+class _Whole:
+    def __init__(self, sim):
+        self.sim = sim
+
+    def state(self):
+        return self.sim.state()
+
+    def counters(self):
+        return self.sim.counters()
+
+
+@pytest.mark.parametrize("K,bias,n", [(1, 0.0, 300), (7, 0.5, 300), (64, 0.0, 1), (16, 0.2, 129), (64, 0.0, 257)])
+def test_precise_rollout_is_a_valid_trajectory(K, bias, n):
+    torch = torch_cuda()
+    T, seed = 64, 4
+    p = inputs.mlp_params(1, bias)
+    sim = binding.Sim(oracle.CARTPOLE, n, 4, seed, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE)
+    out = sim.rollout(T, K, torch.from_numpy(p).cuda())
+    torch.cuda.synchronize()
+    assert sim.device_status() == 0 and sim.launches == 1 + -(-T // K)
+    g = {k: to_np(out[k]) for k in ("obs", "act", "rew", "done")}
+    differ, ambiguous, total = check_precise_rollout(_Whole(sim), g, p, seed, np.arange(n, dtype=np.uint32), T, "precise K%d n%d" % (K, n))
+    assert differ <= 1                                              # 2e4 env-steps at most: a differing action is a 1e-5 event
+    if n >= 100:
+        frac0 = float((out["act"] == 0).float().mean())
+        assert 0.05 < frac0 < 0.95
+        assert int(out["done"].sum()) > 0                           # resets happened inside the window
+
+
+def test_precise_rollout_is_repeatable_k_invariant_and_matches_exact_mode_almost_everywhere():
+    torch = torch_cuda()
+    n, T, seed = 5000, 40, 11
+    p = torch.from_numpy(inputs.mlp_params(3, 0.2)).cuda()
+    a = binding.Sim(oracle.CARTPOLE, n, 4, seed, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE).rollout(T, 40, p)
+    b = binding.Sim(oracle.CARTPOLE, n, 4, seed, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE).rollout(T, 8, p)
+    for k in ("obs", "act", "rew", "done"):
+        assert torch.equal(a[k], b[k]), k                           # same device, same inputs: same bits, whatever K
+    e = binding.Sim(oracle.CARTPOLE, n, 4, seed).rollout(T, 40, p)
+    # 2e5 env-steps: the whole trajectory equals the exact mode's unless a 1e-5 event happened in an env
+    same_envs = int((a["act"] == e["act"]).all(0).sum())
+    assert same_envs >= n - 3, same_envs
+
+
+def test_precise_mode_with_offset_and_mode_switch():
+    torch = torch_cuda()
+    n, T, seed, off = 200, 24, 5, 1000
+    p = inputs.mlp_params(2, 0.1)
+    dp = torch.from_numpy(p).cuda()
+    sim = binding.Sim(oracle.CARTPOLE, n, 4, seed, env_offset=off, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE)
+    out = sim.rollout(T, 5, dp)
+    torch.cuda.synchronize()
+    ids = np.arange(off, off + n, dtype=np.uint32)                  # env ids are global
+    g = {k: to_np(out[k]) for k in ("obs", "act", "rew", "done")}
+    check_precise_rollout(_Whole(sim), g, p, seed, ids, T, "offset")
+    orc = oracle.OracleSim(oracle.CARTPOLE, seed=seed, env_ids=ids)
+    orc.rollout(T, actions=g["act"])
+    binding.sim_set_policy_mode(sim.h, binding.SIM_POLICY_EXACT)    # back to exact mode on the same handle
+    out2 = sim.rollout(10, 10, dp)
+    ref2 = orc.rollout(10, policy_params=p)
+    for k in ("obs", "act", "rew", "done"):
+        assert_same_bits(to_np(out2[k]), ref2[k], "exact after precise " + k)
+    assert sim.device_status() == 0
+    acro = binding.Sim(oracle.ACROBOT, 16)
+    assert binding.lib().sim_set_policy_mode(acro.h, binding.SIM_POLICY_TENSOR_PRECISE) == binding.SIM_EINVAL
+
+
+def test_cfg3_full_size_in_precise_mode():
+    """The largest CartPole + MLP workload in the launch configuration the bench times (one launch of 500 steps over
+    2^20 envs): 1500 sampled envs (first, last, random; 7.5e5 env-steps) are checked by the oracle, differing and
+    ambiguous actions are counted."""
+    torch = torch_cuda()
+    w = inputs.WORKLOADS["cfg3"]
+    ids = inputs.sample_env_ids(29, w.n_envs, 1500)
+    p = inputs.mlp_params(w.mlp_seed)
+    sim = binding.Sim(w.env_kind, w.n_envs, w.state_dim, w.seed, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE)
+    out = sim.rollout(w.T, max(w.k_sweep), torch.from_numpy(p).cuda())
+    torch.cuda.synchronize()
+    assert sim.device_status() == 0
+    sel = torch.from_numpy(ids.astype(np.int64)).cuda()
+    g = {k: to_np(out[k][:, sel]) for k in ("obs", "act", "rew", "done")}
+
+    class View:                                                     # the handle's state and counters restricted to the sample
+        def state(self_):
+            return sim.state()[sel]
+
+        def counters(self_):
+            ep, rc, t = sim.counters()
+            return ep[sel], rc[sel], t
+
+    differ, ambiguous, total = check_precise_rollout(View(), g, p, w.seed, ids, w.T, "cfg3 precise", HARNESS_TOL)
+    print("cfg3 precise: %d of %d sampled env-steps differ from the oracle's action, %d lie inside the ambiguity margin" % (differ, total, ambiguous))
+    assert differ <= 1e-5 * total, (differ, total)
+    assert ambiguous <= 1e-5 * total, (ambiguous, total)            # the margin of the harness weights covers 3.4e-6 of the unit interval
+    # properties that hold at any size
+    ep, rc, t = sim.counters()
+    assert torch.equal(out["done"].sum(0, dtype=torch.int32), rc)
+    assert float(out["obs"][:, :, 0].abs().max()) <= float(np.float32(2.4)) and float(out["obs"][:, :, 2].abs().max()) <= 0.2095
+    # against the exact kernel at full size: the first steps agree in all but a 1e-5 fraction of the envs
+    exact = binding.Sim(w.env_kind, w.n_envs, w.state_dim, w.seed)
+    ref = exact.rollout(4, 4, torch.from_numpy(p).cuda(), want=("act",))
+    mism = int((out["act"][:4] != ref["act"]).any(0).sum())
+    print("cfg3 precise vs exact kernel, first 4 steps of 2^20 envs: %d envs differ" % mism)
+    assert mism <= 4 * 1e-5 * w.n_envs + 8, mism
