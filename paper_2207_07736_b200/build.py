@@ -41,7 +41,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     def compile_one(src):
         obj = objdir / (src[:-3] + ".o")
         if force or _stale(obj, [CSRC / src, *headers]):
-            cmd = [nvcc, *NVCC_FLAGS, *( ["-Xptxas", "-v"] if verbose else []), "-c", str(CSRC / src), "-o", str(obj)]
+            cmd = [nvcc, *NVCC_FLAGS, *os.environ.get("SIM_EXTRA_NVCC_FLAGS", "").split(), *(["-Xptxas", "-v"] if verbose else []), "-c", str(CSRC / src), "-o", str(obj)]
             r = subprocess.run(cmd, capture_output=True, text=True)
             if verbose or r.returncode:
                 sys.stderr.write(r.stdout + r.stderr)

@@ -215,13 +215,27 @@ __device__ __forceinline__ bool contract(Smem &s, Ctx &c, uint32_t *status)
     return true;
 }
 
-// tanh of two values given y = 2 log2(e) z: 1 - 2 / (2^y + 1).  Saturates correctly: 2^y = inf gives 1, 2^y = 0 gives -1.
+// tanh of two values given y = 2 log2(e) z: 1 - 2 / (2^y + 1).  The special-function unit is the busiest pipe of
+// this kernel, so the two reciprocals share ONE hardware reciprocal: r = 1 / (da db), 1/da = r db, 1/db = r da.
+// y is clamped to 60 first (tanh is 1 to the last bit long before: 2 / (2^60 + 1) < 2^-58), so that da db stays
+// finite; 2^y = 0 for very negative y gives d = 1 and tanh = -1 as it should.
+#ifndef TCP_PAIRED_RCP
+#define TCP_PAIRED_RCP 1
+#endif
 __device__ __forceinline__ f2 tanh2_from_scaled(f2 y)
 {
-    const f2 e = pk(ex2_approx(lo(y)), ex2_approx(hi(y)));
+#if TCP_PAIRED_RCP
+    const f2 e = pk(ex2_approx(fminf(lo(y), 60.0f)), ex2_approx(fminf(hi(y), 60.0f)));
+    const f2 d = add2(e, splat(1.0f));
+    const float r = rcp_approx(__fmul_rn(lo(d), hi(d)));
+    const f2 q = mul2(splat(r), pk(hi(d), lo(d)));                    // (1 / da, 1 / db)
+    return fma2(splat(-2.0f), q, splat(1.0f));
+#else
+    const f2 e = pk(ex2_approx(lo(y)), ex2_approx(hi(y)));            // saturates by itself: 2^y = inf gives 1
     const f2 d = add2(e, splat(1.0f));
     const f2 r = pk(rcp_approx(lo(d)), rcp_approx(hi(d)));
     return fma2(splat(-2.0f), r, splat(1.0f));
+#endif
 }
 
 // Four activations -> four hi parts (cut to 11 bits, exact in FP16) and four lo parts, packed.
