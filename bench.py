@@ -329,13 +329,41 @@ def sweep_workload(torch, binding, sim, w, n, d_params, out, sampler, peaks, rep
     return sweep
 
 
+def k1_burst(torch, sim, w, sampler, peaks, launches=16, idle_s=1.5):
+    """One-step launches of a state-streaming workload timed as a short burst after an idle pause, i.e. at the clock
+    an unthrottled GPU runs at (the measured HBM copy rate they are compared with is itself a best-of-ten burst).  The
+    sweep's own K = 1 figure is the sustained one: half a second per repetition, by which time the power cap has
+    lowered the SM clock."""
+    hbm_gbs = peaks[0]
+    sim.reset()
+    sim.rollout(4, 1, None, out={})                                      # warm-up launches
+    torch.cuda.synchronize()
+    time.sleep(idle_s)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    sim.rollout(launches, 1, None, out={})
+    e1.record()
+    e1.synchronize()
+    t1 = time.perf_counter()
+    ms = e0.elapsed_time(e1) / launches
+    rate = w.n_envs / (ms * 1e-3)
+    clk = sampler.window(t0, t1) if sampler is not None and sampler.ok else {}
+    return {"launches": launches, "ms_per_launch": ms, "env_steps_per_sec": rate,
+            "hbm_frac": algorithmic_bytes_per_env_step(w, 1) * rate / (hbm_gbs * 1e9), "sm_mhz": clk.get("sm_mhz"), "clock_reasons": clk.get("reasons"),
+            "note": "%d one-step launches after %.1f s idle" % (launches, idle_s)}
+
+
 def side_pass(torch, binding, key, wname, policy_mode, dev, sampler, peaks, reps):
     """One workload of the default run's side passes: its own handle and outputs, freed afterwards."""
     w = inputs.WORKLOADS[wname]
     sim = binding.Sim(w.env_kind, w.n_envs, w.state_dim, w.seed, device=dev, policy_mode=policy_mode_code(binding, policy_mode))
     d_params = None if w.mlp_seed is None else torch.from_numpy(inputs.mlp_params(w.mlp_seed)).to(dev)
     out = sim.alloc_outputs(w.T) if w.trajectory else {}
+    burst = None
     try:
+        if not w.trajectory and 1 in w.k_sweep:
+            burst = k1_burst(torch, sim, w, sampler, peaks)              # first, while the GPU is still cool
         sweep = sweep_workload(torch, binding, sim, w, w.n_envs, d_params, out, sampler, peaks, reps, key, policy_mode)
         status = sim.device_status() if policy_mode != "exact" else 0
     finally:
@@ -347,6 +375,8 @@ def side_pass(torch, binding, key, wname, policy_mode, dev, sampler, peaks, reps
             "trajectory": bool(w.trajectory), "unit": "env-steps/s", "k_sweep": sweep}
     if policy_mode != "exact":
         line["device_status"] = status
+    if burst is not None:
+        line["k1_burst"] = burst
     below = [k for k, v in sweep.items() if v["target_point"] and not v["meets_60pct"]]
     line["target_points_below_60pct"] = below
     return line

@@ -59,10 +59,13 @@ __device__ __forceinline__ void synth_steps(const SynthArgs &a, f2 (&P)[EE / 2],
     for (int b = 0; b < nblk; ++b) {
         uint4 blk = make_uint4(0u, 0u, 0u, 0u);
         if (LEAN || !a.actions) blk = philox(env, a.tb0 + (uint32_t)b, 0u, 0u, a.rk);
+        // steps of this launch inside block b: words jlo..jhi-1 (short chunks unroll all four words and skip by test;
+        // long chunks run a rolled loop over exactly the words in range, which is one iteration for a one-step launch)
+        const int jlo = EE <= 8 ? 0 : max(0, a.phase - 4 * b), jhi = EE <= 8 ? 4 : min(4, a.phase + a.K - 4 * b);
 #pragma unroll(EE <= 8 ? 4 : 1)
-        for (int j4 = 0; j4 < 4; ++j4) {
+        for (int j4 = jlo; j4 < jhi; ++j4) {
             const int k = 4 * b + j4 - a.phase;
-            if (k < 0 || k >= a.K) continue;
+            if (EE <= 8 && (k < 0 || k >= a.K)) continue;
             const uint32_t w = j4 == 0 ? blk.x : j4 == 1 ? blk.y : j4 == 2 ? blk.z : blk.w;
 
             if (!LEAN && a.out_obs && valid) {

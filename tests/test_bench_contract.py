@@ -34,6 +34,30 @@ def test_reference_arm_prints_the_contract_line():
     assert line["e2e"] == {"value": line["value"], "unit": "env-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
 
 
+def test_both_arms_print_the_same_config_keys():
+    """The reference arm's `config` names the workload with the keys (and, for one GPU, the values) the CUDA arm prints."""
+    import argparse
+    w = inputs.WORKLOADS["cfg2"]
+    args = argparse.Namespace(compute_factor=1, action_bits=False, policy_mode="exact")
+    gpu = bench.config_dict(w, w.n_envs, 1000, args, bench.trajectory_bytes(w, w.n_envs), 1)
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "3",
+                          "--cpu-seconds", "0.05"], capture_output=True, text=True, timeout=300, cwd=ROOT)
+    ref = json.loads(out.stdout.strip().splitlines()[-1])["config"]
+    assert ref == gpu
+    assert gpu["trajectory_bytes_per_step"] == 22 * 65536 * 1000
+
+
+def test_roofline_point_picks_the_binding_bound():
+    hbm, fp32 = 6548.8, 74.44992
+    w2, w3, w5 = inputs.WORKLOADS["cfg2"], inputs.WORKLOADS["cfg3"], inputs.WORKLOADS["cfg5_S4096"]
+    p = bench.roofline_point(w2, 1000, 2.5e11, hbm, fp32)
+    assert p["bound"] == "hbm" and abs(p["frac"] - 22.048 * 2.5e11 / 6548.8e9) < 1e-9
+    p = bench.roofline_point(w3, 500, 4.17e9, hbm, fp32)
+    assert p["bound"] == "alu" and abs(p["frac"] - 9121 * 4.17e9 / 74.44992e12) < 1e-9 and p["frac_expanded_ledger"] > p["frac"]
+    assert bench.roofline_point(w5, 1, 1.37e8, hbm, fp32)["bound"] == "hbm"            # state streaming
+    assert bench.roofline_point(w5, 256, 3.4e8, hbm, fp32)["bound"] == "alu"           # fused: the sine
+
+
 def test_reference_arm_other_ranks_do_nothing():
     env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1"],
