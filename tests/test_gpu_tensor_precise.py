@@ -165,6 +165,26 @@ def test_precise_mode_with_offset_and_mode_switch():
     assert binding.lib().sim_set_policy_mode(acro.h, binding.SIM_POLICY_TENSOR_PRECISE) == binding.SIM_EINVAL
 
 
+def test_precise_mode_with_compute_factor_and_host_buffers():
+    """Compute factor C = 3 (three dynamics iterations per recorded step) and the host-buffer entry point."""
+    torch = torch_cuda()
+    n, T, seed = 260, 20, 13
+    p = inputs.mlp_params(4, 0.1)
+    sim = binding.Sim(oracle.CARTPOLE, n, 4, seed, compute_factor=3, policy_mode=binding.SIM_POLICY_TENSOR_PRECISE)
+    h = {"obs": np.zeros((T, n, 4), np.float32), "act": np.zeros((T, n), np.int8), "rew": np.zeros((T, n), np.float32), "done": np.zeros((T, n), np.uint8)}
+    binding.sim_rollout_host(sim.h, T, 6, p, h["obs"], h["act"], h["rew"], h["done"])
+    assert sim.device_status() == 0
+    ids = np.arange(n, dtype=np.uint32)
+    orc = oracle.OracleSim(oracle.CARTPOLE, seed=seed, env_ids=ids, compute_factor=3)
+    ref = orc.rollout(T, actions=h["act"])
+    for k in ("obs", "rew", "done"):
+        assert_same_bits(h[k], ref[k], "C=3 host " + k)
+    assert_same_bits(to_np(sim.state()), orc.state, "C=3 final state")
+    lg = exact_logits(p, h["obs"].reshape(-1, 4))
+    want = np.array([oracle.sample_action(lg[i], oracle.action_word(seed, int(i % n), i // n)) for i in range(T * n)], dtype=np.int8).reshape(T, n)
+    assert int((want != h["act"]).sum()) <= 1
+
+
 def test_cfg3_full_size_in_precise_mode():
     """The largest CartPole + MLP workload in the launch configuration the bench times (one launch of 500 steps over
     2^20 envs): 1500 sampled envs (first, last, random; 7.5e5 env-steps) are checked by the oracle, differing and
