@@ -61,6 +61,7 @@ struct Smem {
     uint4 b2[64 * kChA];             // layer-2 weights: hi[64] | lo[64] per output unit
     uint4 b3[16 * kChB3];            // layer-3 weights: rows W3[0] hi, W3[0] lo, W3[1] hi, W3[1] lo; rows 4..15 zero
     float bias2c[64];                // b2 * 2 log2(e): added as the constant term of the tanh argument
+    float4 w3p[32];                  // output layer in fp32, in the order the four-way tanh delivers h2: entry 2g + u = (W3[0][c], W3[0][c+2], W3[1][c], W3[1][c+2]), c = 4g + u
     float bias3[2];
     uint32_t tmem_slot;              // TMEM base address written by tcgen05.alloc
     uint32_t pad;
@@ -126,6 +127,10 @@ __device__ __forceinline__ void setup(const float *__restrict__ p, Smem &s, Ctx 
         uint16_t hi, lo;
         f16_split(p[4480 + i], hi, lo);
         tc_put(s.b3, 2u * a, k, kChB3, hi); tc_put(s.b3, 2u * a + 1u, k, kChB3, lo);
+    }
+    if (tid < 32u) {
+        const uint32_t c0 = 4u * (tid >> 1) + (tid & 1u);
+        s.w3p[tid] = make_float4(p[4480 + c0], p[4480 + c0 + 2], p[4544 + c0], p[4544 + c0 + 2]);
     }
     if (tid < 2u) s.bias3[tid] = p[4608 + tid];
     if (tid == 0u) {
@@ -238,6 +243,21 @@ __device__ __forceinline__ f2 tanh2_from_scaled(f2 y)
 #endif
 }
 
+// tanh of FOUR values with one hardware reciprocal: yA = (a0, a1), yB = (b0, b1) scaled arguments; returns the
+// transposed pairs T1 = (tanh a0, tanh b0), T2 = (tanh a1, tanh b1).  With d = 2^y + 1: P = (da0 da1, db0 db1), r = 1 / (PA PB),
+// R = r (PB, PA) = (1 / PA, 1 / PB), 1 / d_x0 = R d_x1, 1 / d_x1 = R d_x0.  Arguments are clamped to 30 (tanh is 1 to the last
+// bit from 2^y = 2^26 on), so the product of the four stays finite; 2^y = 0 for very negative y gives d = 1 and tanh = -1.
+__device__ __forceinline__ void tanh4_from_scaled(f2 yA, f2 yB, f2 &T1, f2 &T2)
+{
+    const f2 D1 = add2(pk(ex2_approx(fminf(lo(yA), 30.0f)), ex2_approx(fminf(lo(yB), 30.0f))), splat(1.0f));   // (da0, db0)
+    const f2 D2 = add2(pk(ex2_approx(fminf(hi(yA), 30.0f)), ex2_approx(fminf(hi(yB), 30.0f))), splat(1.0f));   // (da1, db1)
+    const f2 P = mul2(D1, D2);
+    const float r = rcp_approx(__fmul_rn(lo(P), hi(P)));
+    const f2 R = mul2(splat(r), pk(hi(P), lo(P)));
+    T1 = fma2(splat(-2.0f), mul2(R, D2), splat(1.0f));
+    T2 = fma2(splat(-2.0f), mul2(R, D1), splat(1.0f));
+}
+
 // Four activations -> four hi parts (cut to 11 bits, exact in FP16) and four lo parts, packed.
 __device__ __forceinline__ void split_pack(f2 t, uint32_t &hi_pair, uint32_t &lo_pair)
 {
@@ -267,21 +287,70 @@ __device__ __forceinline__ void activate(Smem &s, const Ctx &c)
                 const int col = 32 * half + 16 * q + 8 * h;           // first of these eight columns
                 uint32_t hp[4], lp[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const f2 z = pk(__uint_as_float(v[q][8 * h + 2 * i]), __uint_as_float(v[q][8 * h + 2 * i + 1]));
-                    f2 y;
-                    if (BIAS) {
-                        const float2 b = *reinterpret_cast<const float2 *>(&s.bias2c[col + 2 * i]);
-                        y = fma2(z, scale, pk(b.x, b.y));
-                    } else {
-                        y = mul2(z, scale);
+                for (int i = 0; i < 4; i += 2) {
+                    f2 y[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const f2 z = pk(__uint_as_float(v[q][8 * h + 2 * (i + u)]), __uint_as_float(v[q][8 * h + 2 * (i + u) + 1]));
+                        if (BIAS) {
+                            const float2 b = *reinterpret_cast<const float2 *>(&s.bias2c[col + 2 * (i + u)]);
+                            y[u] = fma2(z, scale, pk(b.x, b.y));
+                        } else {
+                            y[u] = mul2(z, scale);
+                        }
                     }
-                    split_pack(tanh2_from_scaled(y), hp[i], lp[i]);
+                    f2 T1, T2;                                         // (t[c], t[c+2]), (t[c+1], t[c+3]) for c = col + 2 i
+                    tanh4_from_scaled(y[0], y[1], T1, T2);
+                    f2 H1, H2;                                         // hi parts: 11 significant bits, exact in FP16
+                    H1.v = T1.v & 0xFFFFE000FFFFE000ull; H2.v = T2.v & 0xFFFFE000FFFFE000ull;
+                    const f2 L1 = sub2(T1, H1), L2 = sub2(T2, H2);
+                    hp[i] = pack_f16x2(lo(H1), lo(H2)); hp[i + 1] = pack_f16x2(hi(H1), hi(H2));
+                    lp[i] = pack_f16x2(lo(L1), lo(L2)); lp[i + 1] = pack_f16x2(hi(L1), hi(L2));
                 }
                 row[(col >> 3) * 8] = make_uint4(hp[0], hp[1], hp[2], hp[3]);            // chunk index along K: hi part
                 row[(8 + (col >> 3)) * 8] = make_uint4(lp[0], lp[1], lp[2], lp[3]);      // lo part
             }
     }
+}
+
+#ifndef TCP_L3_FP32
+#define TCP_L3_FP32 1
+#endif
+
+// Output layer on the fp32 pipes: my accumulator row of layer 2 -> + bias -> tanh -> logits = b3 + W3 h2, accumulated
+// in packed form (two partial sums per logit, added at the end).  Saves the hi / lo split of h2, its shared-memory
+// stores and the third round trip to the tensor core, and is exact up to fp32 rounding.
+__device__ __forceinline__ f2 activate_output(const Smem &s, const Ctx &c)
+{
+    const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
+    const f2 scale = splat(kTwoLog2e);
+    f2 acc0 = pk(s.bias3[0], 0.0f), acc1 = pk(s.bias3[1], 0.0f);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint32_t v[2][16];
+        tc_load16(taddr + 32u * (uint32_t)half, v[0]);
+        tc_load16(taddr + 32u * (uint32_t)half + 16u, v[1]);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) {
+                const int col = 32 * half + 16 * q + 2 * i;               // columns col .. col + 3
+                f2 y[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const f2 z = pk(__uint_as_float(v[q][2 * (i + u)]), __uint_as_float(v[q][2 * (i + u) + 1]));
+                    const float2 b = *reinterpret_cast<const float2 *>(&s.bias2c[col + 2 * u]);
+                    y[u] = fma2(z, scale, pk(b.x, b.y));
+                }
+                f2 T1, T2;                                                 // (h[col], h[col+2]), (h[col+1], h[col+3])
+                tanh4_from_scaled(y[0], y[1], T1, T2);
+                const float4 wa = s.w3p[col >> 1], wb = s.w3p[(col >> 1) + 1];
+                acc0 = fma2(pk(wa.x, wa.y), T1, acc0); acc1 = fma2(pk(wa.z, wa.w), T1, acc1);
+                acc0 = fma2(pk(wb.x, wb.y), T2, acc0); acc1 = fma2(pk(wb.z, wb.w), T2, acc1);
+            }
+    }
+    return pk(__fadd_rn(lo(acc0), hi(acc0)), __fadd_rn(lo(acc1), hi(acc1)));
 }
 
 // Logits of this thread's observation; the group's 128 threads evaluate their 128 observations together.
@@ -305,6 +374,10 @@ __device__ __forceinline__ bool policy(const float4 o, Smem &s, Ctx &c, uint32_t
     if (!contract<LAYER1>(s, c, status)) return false;
     activate<false>(s, c);
     if (!contract<LAYER2>(s, c, status)) return false;
+#if TCP_L3_FP32
+    logits = activate_output(s, c);
+    return true;
+#endif
     activate<true>(s, c);
     if (!contract<LAYER3>(s, c, status)) return false;
     const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
