@@ -42,8 +42,8 @@ TRAJ_BYTES_S4 = 22          # obs 16 + act 1 + rew 4 + done 1
 # nominal / operation-expanded flops per env-step (fma = 2, any other fp32 op = 1, integer work = 0)
 FLOPS = {"cartpole": (27, 52), "acrobot": (181, 455), "mlp": (9094, 12205)}
 # padded tensor-core contractions of the two tensor policy modes (flop per env-step, FP16 operands)
-TENSOR_FLOPS_PER_ENV_STEP = {"tensor": 2 * (16 * 64 + 80 * 64 + 80 * 16), "tensor_precise": 2 * (16 * 64 + 208 * 64 + 144 * 16)}
-MUFU_PER_ENV_STEP = {"tensor": 128, "tensor_precise": 192}      # special-function instructions per env-step (tanh; or two ex2 and one shared rcp per pair)
+TENSOR_FLOPS_PER_ENV_STEP = {"tensor": 2 * (16 * 64 + 80 * 64 + 80 * 16), "tensor_precise": 2 * (32 * 64 + 192 * 64)}
+MUFU_PER_ENV_STEP = {"tensor": 128, "tensor_precise": 160}      # special-function instructions per env-step (tanh; or one ex2 each and one shared rcp per four)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused rollout kernel, from the ncu
 # captures summarised under profiles/ (keyed by workload and K_fused; other shapes report null)
 NCU_TRAFFIC_BYTES = {("cfg2", 1000): 1.3863e9}

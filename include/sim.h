@@ -107,10 +107,12 @@ int sim_set_action_stream(sim_t *s, int mode);
  *       z1 = W1 obs + b1      observation, W1 and b1 each split into THREE FP16 parts (x = x1 + x2 + x3); the six
  *                             leading products of parts are exact and summed in fp32 by the tensor core
  *       h1 = tanh'(z1)        tanh'(z) = 1 - 2 / (2^(2 log2(e) z) + 1) in fp32 with the GPU's base-2 exponential
- *                             and reciprocal approximations: absolute error below 3e-7
+ *                             and reciprocal approximations (one reciprocal shared by four evaluations): absolute
+ *                             error below 4e-7
  *       z2 = b2 + W2 h1       h1 = hi + lo (hi = h1 cut to 11 significant bits, lo = f16(h1 - hi)), W2 = f16(W2) +
  *                             f16(W2 - f16(W2)); hi*hi + hi*lo + lo*hi summed in fp32 by the tensor core, b2 added in fp32
- *       h2 = tanh'(z2);       logits = b3 + W3 h2 with the same splits.
+ *       h2 = tanh'(z2);       logits = b3 + W3 h2 in fp32 on the ordinary pipes (two partial sums per logit, over the
+ *                             hidden units 4g, 4g+2 and 4g+1, 4g+3, added at the end).
  *   SIM_POLICY_TENSOR: the fast mode; it does NOT meet the 1e-5 logit tolerance (typical logit error 2e-3, bound
  *     below); use it where throughput matters more than the third digit of the action probabilities.
  *       z1 = W1 obs + b1      observation, W1 and b1 each split into two FP16 parts (x = hi + lo); the

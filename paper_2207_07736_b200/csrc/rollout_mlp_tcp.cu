@@ -1,26 +1,28 @@
-// Fused CartPole rollout with the MLP policy in PRECISE TENSOR mode: all three layers of the 4-64-64-2 network run
-// on the 5th-generation tensor cores (tcgen05, FP16 operands, fp32 accumulators in TMEM), but every operand is
-// carried as a sum of FP16 parts whose products are exact, and tanh is evaluated in fp32, so that the logits stay
-// within 1e-5 of the fp32 definition (the fast tensor mode of rollout_mlp_tc.cu trades three more digits for speed).
-// The paper names fusing simulation and inference as future work (Section 7); this is that fusion at fp32-level accuracy.
+// Fused CartPole rollout with the MLP policy in PRECISE TENSOR mode: the two hidden layers of the 4-64-64-2 network
+// run on the 5th-generation tensor cores (tcgen05, FP16 operands, fp32 accumulators in TMEM), but every operand is
+// carried as a sum of FP16 parts whose products are exact, tanh is evaluated in fp32 and the two-unit output layer
+// runs on the fp32 pipes, so that the logits stay within 1e-5 of the fp32 definition (the fast tensor mode of
+// rollout_mlp_tc.cu trades three more digits for speed).  The paper names fusing simulation and inference as future
+// work (Section 7); this is that fusion at fp32-level accuracy.
 //
 // One CTA = kGroups groups of 128 threads; a group owns one tile of 128 envs (thread = env = row of the operand tile
 // = TMEM lane of the accumulator) and synchronises on its own named barrier and its own mbarrier, so the groups
 // drift apart and one converts while another's contraction runs.  The weight tiles are shared by the groups.
-// Per step and tile, three contractions, each issued by the group's first thread and awaited through the mbarrier:
+// Per step and tile, two contractions, each issued by the group's first thread and awaited through the mbarrier:
 //   1. z1[128x64] = A1[128x32] B1^T: observation o = o1 + o2 + o3 and W1 = w1 + w2 + w3 (b1 likewise) in three
 //      FP16 parts; the columns pair the parts so that o1w1 + o2w1 + o3w1 + o1w2 + o2w2 + o1w3 + b1 is summed (what is
 //      dropped is below 2^-33 of a product);
 //   2. z2[128x64] = Ahi Bhi^T + Ahi Blo^T + Alo Bhi^T with h1 = hi + lo (hi = h1 cut to 11 bits, lo = f16(h1 - hi)),
 //      W2 = f16(W2) + f16(W2 - f16(W2)); twelve instructions of K = 16 into one accumulator; b2 is added in fp32
-//      when the accumulator row is read back;
-//   3. l[128x16] = Ahi B3^T + Alo B3^T with B3 rows (W3[0] hi, W3[0] lo, W3[1] hi, W3[1] lo): logit i = l[2i] +
-//      l[2i+1] + b3[i].
+//      when the accumulator row is read back.
+// Each thread turns its accumulator row of layer 1 into its operand row of layer 2 (tcgen05.ld, tanh, hi / lo split,
+// sixteen 16-byte shared-memory stores) and its accumulator row of layer 2 straight into the two logits
+// (tanh, then logit_i = b3[i] + sum_j W3[i][j] h2[j] in fp32, two packed partial sums per logit); then it samples,
+// steps the physics, resets and stores exactly like the exact kernel.  An output layer on the tensor core (a third
+// contraction with N = 16) was measured 13 % slower: it needs the split of h2, its stores and a third round trip.
 // tanh(z) = 1 - 2 / (2^(2 log2(e) z) + 1) with the hardware's base-2 exponential and reciprocal approximations
-// (relative error about 2^-22 each): absolute error below 3e-7.
-// Each thread converts its own accumulator row (tcgen05.ld, 32 lanes x 32 bit) into the next operand row, then
-// samples, steps the physics, resets and stores exactly like the exact kernel.  A1 lives in the first 8 KB of the
-// tile's operand buffer (it is dead before h1 is written).
+// (relative error about 2^-22 each), four evaluations sharing one reciprocal: absolute error below 4e-7.
+// A1 lives in the first 8 KB of the tile's operand buffer (it is dead before h1 is written).
 // Every wait is bounded: when a barrier does not complete in time the group records bit 0 in the status word and
 // skips its remaining steps; the CTA then frees its TMEM columns and returns.
 #include <mutex>
@@ -44,14 +46,12 @@ constexpr int kThreads = 128 * kGroups;
 constexpr uint32_t kTile = 128u;                  // envs (rows) per tile = threads per group
 constexpr uint32_t kChA = 16u;                    // 16-byte chunks per operand row of layers 2 and 3: h hi[64] | h lo[64]
 constexpr uint32_t kCh1 = 4u;                     // layer-1 operand row: 32 FP16 values
-constexpr uint32_t kChB3 = 8u;                    // layer-3 weight rows: 64 FP16 values
-constexpr uint32_t kTileCols = 64u;               // TMEM columns (fp32) per tile: z1 / z2 use all, the logits the first 16
+constexpr uint32_t kTileCols = 64u;               // TMEM columns (fp32) per tile
 constexpr uint32_t kCols = kGroups * kTileCols <= 32 ? 32u : kGroups * kTileCols <= 64 ? 64u : kGroups * kTileCols <= 128 ? 128u
                            : kGroups * kTileCols <= 256 ? 256u : 512u;      // allocations are powers of two
 static_assert(kGroups >= 1 && kGroups * kTileCols <= 512, "a CTA's tiles must fit the 512 TMEM columns of an SM");
 // Instruction descriptors: D = fp32 (bit 4), A = B = FP16 (0 at bits 7 and 10), K-major, N >> 3 (bit 17), M >> 4 (bit 24).
 constexpr uint32_t kIdescN64 = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescN16 = (1u << 4) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr long long kWaitCycles = 2000000000ll;   // about a second at the SM clock
 constexpr float kTwoLog2e = 2.8853900817779268f;  // 2 log2(e)
 
@@ -59,7 +59,6 @@ struct Smem {
     uint4 a[kGroups][kTile * kChA];  // per tile: operand rows (h hi | h lo), 32 KB; the layer-1 rows in its first 8 KB
     uint4 b1[64 * kCh1];             // layer-1 weights and bias, three FP16 parts paired with the observation's
     uint4 b2[64 * kChA];             // layer-2 weights: hi[64] | lo[64] per output unit
-    uint4 b3[16 * kChB3];            // layer-3 weights: rows W3[0] hi, W3[0] lo, W3[1] hi, W3[1] lo; rows 4..15 zero
     float bias2c[64];                // b2 * 2 log2(e): added as the constant term of the tanh argument
     float4 w3p[32];                  // output layer in fp32, in the order the four-way tanh delivers h2: entry 2g + u = (W3[0][c], W3[0][c+2], W3[1][c], W3[1][c+2]), c = 4g + u
     float bias3[2];
@@ -101,7 +100,7 @@ __device__ __forceinline__ bool group_sync_or(uint32_t group, bool flag)
 __device__ __forceinline__ void setup(const float *__restrict__ p, Smem &s, Ctx &c)
 {
     const uint32_t tid = threadIdx.x;
-    constexpr uint32_t weight_chunks = 64u * kCh1 + 64u * kChA + 16u * kChB3;    // b1, b2, b3 are contiguous
+    constexpr uint32_t weight_chunks = 64u * kCh1 + 64u * kChA;    // b1 and b2 are contiguous
     for (uint32_t i = tid; i < weight_chunks; i += kThreads) s.b1[i] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     for (uint32_t i = tid; i < 256u; i += kThreads) {               // W1[j][k]: columns (w1 w1 w1 w2 w2 w3) x 4
@@ -121,12 +120,6 @@ __device__ __forceinline__ void setup(const float *__restrict__ p, Smem &s, Ctx 
         uint16_t hi, lo;
         f16_split(p[320 + i], hi, lo);
         tc_put(s.b2, i >> 6, i & 63u, kChA, hi); tc_put(s.b2, i >> 6, 64u + (i & 63u), kChA, lo);
-    }
-    for (uint32_t i = tid; i < 128u; i += kThreads) {               // W3[a][k] -> rows 2a (hi), 2a+1 (lo)
-        const uint32_t a = i >> 6, k = i & 63u;
-        uint16_t hi, lo;
-        f16_split(p[4480 + i], hi, lo);
-        tc_put(s.b3, 2u * a, k, kChB3, hi); tc_put(s.b3, 2u * a + 1u, k, kChB3, lo);
     }
     if (tid < 32u) {
         const uint32_t c0 = 4u * (tid >> 1) + (tid & 1u);
@@ -162,7 +155,7 @@ __device__ __forceinline__ void teardown(Smem &s)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(s.tmem_slot), "r"(kCols) : "memory");
 }
 
-enum : int { LAYER1 = 0, LAYER2 = 1, LAYER3 = 2 };
+enum : int { LAYER1 = 0, LAYER2 = 1 };
 
 __device__ __forceinline__ void mma_f16(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, bool accumulate)
 {
@@ -190,7 +183,7 @@ __device__ __forceinline__ bool contract(Smem &s, Ctx &c, uint32_t *status)
 #pragma unroll
             for (uint32_t k = 0; k < 2u; ++k)
                 mma_f16(c.tmem, tc_desc(a_addr + k * slice, kCh1), tc_desc(b_addr + k * slice, kCh1), kIdescN64, k != 0u);
-        } else if (LAYER == LAYER2) {
+        } else {
             const uint32_t b_addr = smem_u32(s.b2);
 #pragma unroll
             for (uint32_t k = 0; k < 4u; ++k) {                       // the small terms first, the leading one last
@@ -202,14 +195,6 @@ __device__ __forceinline__ bool contract(Smem &s, Ctx &c, uint32_t *status)
 #pragma unroll
             for (uint32_t k = 0; k < 4u; ++k)
                 mma_f16(c.tmem, tc_desc(a_addr + k * slice, kChA), tc_desc(b_addr + k * slice, kChA), kIdescN64, true);
-        } else {
-            const uint32_t b_addr = smem_u32(s.b3);
-#pragma unroll
-            for (uint32_t k = 0; k < 4u; ++k)
-                mma_f16(c.tmem, tc_desc(a_addr + (4u + k) * slice, kChA), tc_desc(b_addr + k * slice, kChB3), kIdescN16, k != 0u);
-#pragma unroll
-            for (uint32_t k = 0; k < 4u; ++k)
-                mma_f16(c.tmem, tc_desc(a_addr + k * slice, kChA), tc_desc(b_addr + k * slice, kChB3), kIdescN16, true);
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
     }
@@ -220,30 +205,8 @@ __device__ __forceinline__ bool contract(Smem &s, Ctx &c, uint32_t *status)
     return true;
 }
 
-// tanh of two values given y = 2 log2(e) z: 1 - 2 / (2^y + 1).  The special-function unit is the busiest pipe of
-// this kernel, so the two reciprocals share ONE hardware reciprocal: r = 1 / (da db), 1/da = r db, 1/db = r da.
-// y is clamped to 60 first (tanh is 1 to the last bit long before: 2 / (2^60 + 1) < 2^-58), so that da db stays
-// finite; 2^y = 0 for very negative y gives d = 1 and tanh = -1 as it should.
-#ifndef TCP_PAIRED_RCP
-#define TCP_PAIRED_RCP 1
-#endif
-__device__ __forceinline__ f2 tanh2_from_scaled(f2 y)
-{
-#if TCP_PAIRED_RCP
-    const f2 e = pk(ex2_approx(fminf(lo(y), 60.0f)), ex2_approx(fminf(hi(y), 60.0f)));
-    const f2 d = add2(e, splat(1.0f));
-    const float r = rcp_approx(__fmul_rn(lo(d), hi(d)));
-    const f2 q = mul2(splat(r), pk(hi(d), lo(d)));                    // (1 / da, 1 / db)
-    return fma2(splat(-2.0f), q, splat(1.0f));
-#else
-    const f2 e = pk(ex2_approx(lo(y)), ex2_approx(hi(y)));            // saturates by itself: 2^y = inf gives 1
-    const f2 d = add2(e, splat(1.0f));
-    const f2 r = pk(rcp_approx(lo(d)), rcp_approx(hi(d)));
-    return fma2(splat(-2.0f), r, splat(1.0f));
-#endif
-}
-
-// tanh of FOUR values with one hardware reciprocal: yA = (a0, a1), yB = (b0, b1) scaled arguments; returns the
+// tanh of FOUR values given y = 2 log2(e) z: 1 - 2 / (2^y + 1).  The special-function unit is the busiest pipe of this
+// kernel, so the four reciprocals share ONE hardware reciprocal.  yA = (a0, a1), yB = (b0, b1) scaled arguments; returns the
 // transposed pairs T1 = (tanh a0, tanh b0), T2 = (tanh a1, tanh b1).  With d = 2^y + 1: P = (da0 da1, db0 db1), r = 1 / (PA PB),
 // R = r (PB, PA) = (1 / PA, 1 / PB), 1 / d_x0 = R d_x1, 1 / d_x1 = R d_x0.  Arguments are clamped to 30 (tanh is 1 to the last
 // bit from 2^y = 2^26 on), so the product of the four stays finite; 2^y = 0 for very negative y gives d = 1 and tanh = -1.
@@ -258,17 +221,8 @@ __device__ __forceinline__ void tanh4_from_scaled(f2 yA, f2 yB, f2 &T1, f2 &T2)
     T2 = fma2(splat(-2.0f), mul2(R, D1), splat(1.0f));
 }
 
-// Four activations -> four hi parts (cut to 11 bits, exact in FP16) and four lo parts, packed.
-__device__ __forceinline__ void split_pack(f2 t, uint32_t &hi_pair, uint32_t &lo_pair)
-{
-    f2 h; h.v = t.v & 0xFFFFE000FFFFE000ull;
-    const f2 l = sub2(t, h);
-    hi_pair = pack_f16x2(lo(h), hi(h));
-    lo_pair = pack_f16x2(lo(l), hi(l));
-}
-
-// My accumulator row (64 columns) -> (+ bias) -> tanh -> hi / lo FP16 parts -> my row of the group's operand tile.
-template <bool BIAS>
+// My accumulator row of layer 1 (64 columns; b1 is already in it) -> tanh -> hi / lo FP16 parts -> my row of the group's
+// operand tile for layer 2.
 __device__ __forceinline__ void activate(Smem &s, const Ctx &c)
 {
     const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
@@ -292,12 +246,7 @@ __device__ __forceinline__ void activate(Smem &s, const Ctx &c)
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const f2 z = pk(__uint_as_float(v[q][8 * h + 2 * (i + u)]), __uint_as_float(v[q][8 * h + 2 * (i + u) + 1]));
-                        if (BIAS) {
-                            const float2 b = *reinterpret_cast<const float2 *>(&s.bias2c[col + 2 * (i + u)]);
-                            y[u] = fma2(z, scale, pk(b.x, b.y));
-                        } else {
-                            y[u] = mul2(z, scale);
-                        }
+                        y[u] = mul2(z, scale);
                     }
                     f2 T1, T2;                                         // (t[c], t[c+2]), (t[c+1], t[c+3]) for c = col + 2 i
                     tanh4_from_scaled(y[0], y[1], T1, T2);
@@ -312,10 +261,6 @@ __device__ __forceinline__ void activate(Smem &s, const Ctx &c)
             }
     }
 }
-
-#ifndef TCP_L3_FP32
-#define TCP_L3_FP32 1
-#endif
 
 // Output layer on the fp32 pipes: my accumulator row of layer 2 -> + bias -> tanh -> logits = b3 + W3 h2, accumulated
 // in packed form (two partial sums per logit, added at the end).  Saves the hi / lo split of h2, its shared-memory
@@ -372,20 +317,9 @@ __device__ __forceinline__ bool policy(const float4 o, Smem &s, Ctx &c, uint32_t
         row[24] = make_uint4(0x3C003C00u, 0x00003C00u, 0u, 0u);
     }
     if (!contract<LAYER1>(s, c, status)) return false;
-    activate<false>(s, c);
+    activate(s, c);
     if (!contract<LAYER2>(s, c, status)) return false;
-#if TCP_L3_FP32
     logits = activate_output(s, c);
-    return true;
-#endif
-    activate<true>(s, c);
-    if (!contract<LAYER3>(s, c, status)) return false;
-    const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
-    uint32_t l0, l1, l2, l3;
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(l0), "=r"(l1), "=r"(l2), "=r"(l3) : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-    logits = pk(__fadd_rn(__fadd_rn(__uint_as_float(l0), __uint_as_float(l1)), s.bias3[0]),
-                __fadd_rn(__fadd_rn(__uint_as_float(l2), __uint_as_float(l3)), s.bias3[1]));
     return true;
 }
 
