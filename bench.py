@@ -354,6 +354,39 @@ def k1_burst(torch, sim, w, sampler, peaks, launches=16, idle_s=1.5):
             "note": "%d one-step launches after %.1f s idle" % (launches, idle_s)}
 
 
+def k1_graph(torch, sim, w, d_params, out, reps=7):
+    """The launch-bound one-step-per-launch rollout replayed from a CUDA graph that the CALLER captures: the library's
+    calls only enqueue kernels on the handle's stream, so reset + T one-step launches record into one graph."""
+    st = torch.cuda.Stream(device=sim.device)
+    prev = sim.stream
+    sim.use_stream(st)
+    try:
+        with torch.cuda.stream(st):
+            sim.reset()
+            sim.rollout(w.T, 1, d_params, out=out)
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            sim.reset()
+            sim.rollout(w.T, 1, d_params, out=out)
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(st):
+                e0.record()
+                g.replay()
+                e1.record()
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ms = statistics.median(ts)
+        return {"ms": ms, "ms_min": min(ts), "reps": reps, "launches": w.T + 1, "us_per_launch": ms * 1e3 / (w.T + 1),
+                "env_steps_per_sec": w.n_envs * w.T / (ms * 1e-3), "note": "reset + T one-step launches captured once by the caller, replayed"}
+    except Exception as e:                                               # capture is the caller's feature, not the library's: report and go on
+        return {"unavailable": "%s: %s" % (type(e).__name__, e)}
+    finally:
+        sim.use_stream(prev)
+
+
 def side_pass(torch, binding, key, wname, policy_mode, dev, sampler, peaks, reps):
     """One workload of the default run's side passes: its own handle and outputs, freed afterwards."""
     w = inputs.WORKLOADS[wname]
@@ -366,6 +399,7 @@ def side_pass(torch, binding, key, wname, policy_mode, dev, sampler, peaks, reps
             burst = k1_burst(torch, sim, w, sampler, peaks)              # first, while the GPU is still cool
         sweep = sweep_workload(torch, binding, sim, w, w.n_envs, d_params, out, sampler, peaks, reps, key, policy_mode)
         status = sim.device_status() if policy_mode != "exact" else 0
+        graph = k1_graph(torch, sim, w, d_params, out) if key == "cfg1" else None
     finally:
         sim.close()
         del out
@@ -377,6 +411,8 @@ def side_pass(torch, binding, key, wname, policy_mode, dev, sampler, peaks, reps
         line["device_status"] = status
     if burst is not None:
         line["k1_burst"] = burst
+    if graph is not None:
+        line["k1_cuda_graph"] = graph
     below = [k for k, v in sweep.items() if v["target_point"] and not v["meets_60pct"]]
     line["target_points_below_60pct"] = below
     return line

@@ -18,6 +18,11 @@
  *     reset_count [N] u32) are owned by the library: sim_create allocates, sim_destroy frees.
  *   - Except sim_create / sim_destroy / sim_rollout_host, calls only enqueue work on the
  *     handle's stream and return; the caller synchronises the stream.
+ *   - Because those calls only enqueue kernels (no allocation, no synchronisation, no host-side read of device
+ *     data), a caller may record them into a CUDA graph by stream capture and replay it, e.g. sim_reset followed by
+ *     a sim_rollout with K_fused = 1, whose launches are then replayed without per-launch host cost.  The launch
+ *     arguments carry the handle's step counter t as it was at capture time, so a replay repeats exactly the
+ *     captured steps; the host-side t does not advance on replay (set it with sim_set_counters if needed).
  *   - A handle belongs to the CUDA device that was current in sim_create; a call made while
  *     another device is current returns SIM_ESTATE and enqueues nothing.
  *   - All floating point is IEEE binary32 with a fixed operation order, so results are

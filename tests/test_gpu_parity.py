@@ -387,3 +387,34 @@ def test_argument_errors_with_live_handle():
     assert L.sim_set_env_offset(sim.h, (1 << 32) - 8) == binding.SIM_EINVAL
     ep, rc, t = sim.counters()
     assert t == 0                                         # nothing above advanced the handle
+
+
+def test_rollout_records_into_a_cuda_graph_captured_by_the_caller():
+    """The calls only enqueue kernels on the handle's stream, so a caller can capture reset + a one-step-per-launch
+    rollout in a CUDA graph and replay it: every replay writes the oracle's trajectory again."""
+    torch = torch_cuda()
+    w = inputs.WORKLOADS["cfg1"]
+    sim = binding.Sim(w.env_kind, w.n_envs, w.state_dim, w.seed)
+    out = sim.alloc_outputs(w.T)
+    st = torch.cuda.Stream()
+    sim.use_stream(st)
+    with torch.cuda.stream(st):
+        sim.rollout(3, 1, None, out=sim.alloc_outputs(3))          # module loading and the first launches happen outside the capture
+    st.synchronize()
+    launches0 = sim.launches
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        sim.reset()
+        sim.rollout(w.T, 1, None, out=out)
+    assert sim.launches - launches0 == 1 + w.T                     # one graph node per launch
+    orc = oracle.OracleSim(w.env_kind, w.n_envs, w.state_dim, seed=w.seed)
+    ref = orc.rollout(w.T)
+    for replay in range(2):
+        for t in out.values():
+            t.fill_(99)
+        with torch.cuda.stream(st):
+            g.replay()
+        st.synchronize()
+        for k in ("obs", "act", "rew", "done"):
+            assert_same_bits(to_np(out[k]), ref[k], "graph replay %d %s" % (replay, k))
+        assert_same_bits(to_np(sim.state()), orc.state, "state after replay")
