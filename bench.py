@@ -50,6 +50,7 @@ NCU_TRAFFIC_BYTES = {("cfg2", 1000): 1.3863e9}
 # tensor-mode policy: captured on a reduced cfg3 (N = 262 144, T = 100: 533.19 MB for 2.62e7 env-steps) and scaled
 # to the full launch by env-steps (the traffic is the trajectory, proportional to env-steps)
 NCU_TRAFFIC_BYTES_TENSOR = {("cfg3", 500): 533.19e6 / 2.62144e7 * (1048576 * 500)}
+NCU_TRAFFIC_BYTES_TENSOR_PRECISE = {("cfg3", 500): 532.45e6 / 2.62144e7 * (1048576 * 500)}   # same reduced case, precise tensor mode
 POLICY_MODES = ("exact", "tensor", "tensor_precise")
 # the side passes of the default run: (key, workload, policy mode)
 SIDE_PASSES = (("cfg1", "cfg1", "exact"), ("cfg3", "cfg3", "exact"), ("cfg3_tensor", "cfg3", "tensor"),
@@ -546,7 +547,8 @@ def run_gpu(args, w):
     roofline["sampled_sm_mhz"] = clocks["sm_mhz"]
     roofline["meets_60pct"] = bool(roofline["frac"] >= 0.6)
     if roofline["traffic"] is None:
-        table = NCU_TRAFFIC_BYTES_TENSOR if (args.policy_mode == "tensor" and w.mlp_seed is not None) else NCU_TRAFFIC_BYTES if args.policy_mode == "exact" else {}
+        table = NCU_TRAFFIC_BYTES if (args.policy_mode == "exact" or w.mlp_seed is None) else \
+            NCU_TRAFFIC_BYTES_TENSOR if args.policy_mode == "tensor" else NCU_TRAFFIC_BYTES_TENSOR_PRECISE
         full = inputs.WORKLOADS.get(w.name)                          # None for a reduced (profiling) shape
         roofline["traffic"] = table.get((w.name, K)) if full is not None and n == full.n_envs and w.T == full.T else None
     roofline["kernel"] = "fused rollout kernel, K_fused=%d, %d launch(es) per step" % (K, launches_per_step)
