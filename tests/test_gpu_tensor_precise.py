@@ -216,9 +216,16 @@ def test_cfg3_full_size_in_precise_mode():
     ep, rc, t = sim.counters()
     assert torch.equal(out["done"].sum(0, dtype=torch.int32), rc)
     assert float(out["obs"][:, :, 0].abs().max()) <= float(np.float32(2.4)) and float(out["obs"][:, :, 2].abs().max()) <= 0.2095
-    # against the exact kernel at full size: the first steps agree in all but a 1e-5 fraction of the envs
+    # Against the exact kernel over the WHOLE run (its actions are the oracle's, bit for bit: test_cfg3_mlp_full).  Until an
+    # env's first differing action both kernels see identical observations, so that first difference is exactly one
+    # "differing action" event and every step before it one agreeing env-step: rate = events / env-steps compared.
     exact = binding.Sim(w.env_kind, w.n_envs, w.state_dim, w.seed)
-    ref = exact.rollout(4, 4, torch.from_numpy(p).cuda(), want=("act",))
-    mism = int((out["act"][:4] != ref["act"]).any(0).sum())
-    print("cfg3 precise vs exact kernel, first 4 steps of 2^20 envs: %d envs differ" % mism)
-    assert mism <= 4 * 1e-5 * w.n_envs + 8, mism
+    ref = exact.rollout(w.T, max(w.k_sweep), torch.from_numpy(p).cuda(), want=("act",))
+    differs = out["act"] != ref["act"]                                                   # [T, N]
+    any_diff = differs.any(0)
+    first = torch.where(any_diff, differs.to(torch.int8).argmax(0), torch.full_like(any_diff, w.T, dtype=torch.int64))
+    events = int(any_diff.sum())
+    compared = int(first.sum()) + events                                                  # agreeing steps + the differing ones
+    print("cfg3 precise vs exact kernel over %d comparable env-steps of 2^20 envs: %d differing actions (rate %.2e)" % (compared, events, events / compared))
+    assert events <= 1e-5 * compared, (events, compared)
+    assert compared > 0.99 * w.n_envs * w.T                                               # nearly every env-step was comparable
