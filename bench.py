@@ -419,6 +419,22 @@ def side_pass(torch, binding, key, wname, policy_mode, dev, sampler, peaks, reps
     return line
 
 
+def compact_summary(workloads, headline_key, headline_sweep):
+    """One short string per workload: `K<k>=<env-steps/s>/<fraction of the binding roofline>`, with `*` after a point the
+    60 % target is stated for that meets it and `!` after one that misses it.  Short enough to sit at the very end of the
+    headline line, where a truncated record of the output still shows every workload."""
+    def one(key, sweep):
+        parts = []
+        for k, v in sweep.items():
+            mark = ("*" if v["meets_60pct"] else "!") if v.get("target_point") else ""
+            parts.append("K%s=%.3g/%.2f%s" % (k, v["env_steps_per_sec"], v["frac"], mark))
+        return key + " " + " ".join(parts)
+    out = [one(key, line["k_sweep"]) for key, line in workloads.items()]
+    if headline_sweep:
+        out.append(one(headline_key, headline_sweep))
+    return out
+
+
 def run_gpu(args, w):
     import torch
     from paper_2207_07736_b200 import binding
@@ -630,6 +646,11 @@ def run_gpu(args, w):
     if workloads:
         line["workloads"] = workloads
         line["target_points_below_60pct"] = {k: v["target_points_below_60pct"] for k, v in workloads.items() if v["target_points_below_60pct"]}
+    summary = compact_summary(workloads, w.name, sweep)
+    if summary:
+        roofline["all_workloads"] = summary                              # also beside the headline's own roofline
+        line["summary"] = summary                                        # last key: the end of the line names every workload
+        line["summary_legend"] = "K<k_fused>=<env-steps/s>/<fraction of the binding roofline: max(bytes/HBM, nominal flops/fp32)>; * target point >= 0.6, ! target point below"
     print(json.dumps(line), flush=True)
     return 0
 
