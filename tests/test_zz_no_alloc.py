@@ -67,16 +67,19 @@ def test_noalloc_calls_after_the_first_allocate_nothing():
     n, T = 3000, 16
     obs, act, rew, done = _outputs(torch, T, n, 4)
     stream = torch.cuda.current_stream().cuda_stream
-    binding.sim_rollout_noalloc(binding.SIM_CARTPOLE, n, 4, 1, T, 4, None, obs, act, rew, done, stream)     # warm-up call
+    cases = ((binding.SIM_CARTPOLE, 4, 4), (binding.SIM_ACROBOT, 4, 8), (binding.SIM_CARTPOLE, 4, 16))
+    for kind, S, k in cases:                                        # warm-up: address lookup, and each kernel launched once
+        binding.sim_rollout_noalloc(kind, n, S, 1, T, k, None, obs, act, rew, done, stream)
     torch.cuda.synchronize()
     free0, _ = torch.cuda.mem_get_info()
     alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
-    for kind, S, k in ((binding.SIM_CARTPOLE, 4, 4), (binding.SIM_ACROBOT, 4, 8), (binding.SIM_CARTPOLE, 4, 16)):
-        binding.sim_rollout_noalloc(kind, n, S, 2, T, k, None, obs, act, rew, done, stream)
-        torch.cuda.synchronize()
-        free1, _ = torch.cuda.mem_get_info()
-        assert free1 == free0, (kind, free0, free1)
-        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    for seed in (2, 3):
+        for kind, S, k in cases:
+            binding.sim_rollout_noalloc(kind, n, S, seed, T, k, None, obs, act, rew, done, stream)
+            torch.cuda.synchronize()
+            free1, _ = torch.cuda.mem_get_info()
+            assert free1 == free0, (kind, free0, free1)
+            assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
 
 
 def test_noalloc_rejects_what_does_not_fit():
