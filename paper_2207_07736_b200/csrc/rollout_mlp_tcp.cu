@@ -44,7 +44,7 @@ namespace tcp {
 constexpr int kGroups = TCP_GROUPS;               // tiles (groups of 128 threads) per CTA
 constexpr int kThreads = 128 * kGroups;
 constexpr uint32_t kTile = 128u;                  // envs (rows) per tile = threads per group
-constexpr uint32_t kChA = 16u;                    // 16-byte chunks per operand row of layers 2 and 3: h hi[64] | h lo[64]
+constexpr uint32_t kChA = 16u;                    // 16-byte chunks per operand row of layer 2: h1 hi[64] | h1 lo[64]
 constexpr uint32_t kCh1 = 4u;                     // layer-1 operand row: 32 FP16 values
 constexpr uint32_t kTileCols = 64u;               // TMEM columns (fp32) per tile
 constexpr uint32_t kCols = kGroups * kTileCols <= 32 ? 32u : kGroups * kTileCols <= 64 ? 64u : kGroups * kTileCols <= 128 ? 128u
@@ -263,8 +263,8 @@ __device__ __forceinline__ void activate(Smem &s, const Ctx &c)
 }
 
 // Output layer on the fp32 pipes: my accumulator row of layer 2 -> + bias -> tanh -> logits = b3 + W3 h2, accumulated
-// in packed form (two partial sums per logit, added at the end).  Saves the hi / lo split of h2, its shared-memory
-// stores and the third round trip to the tensor core, and is exact up to fp32 rounding.
+// in packed form (two partial sums per logit, added at the end).  Compared with a third contraction this saves the hi / lo
+// split of h2, its shared-memory stores and one more round trip to the tensor core, and is exact up to fp32 rounding.
 __device__ __forceinline__ f2 activate_output(const Smem &s, const Ctx &c)
 {
     const uint32_t taddr = c.tmem + ((c.row & ~31u) << 16);
