@@ -58,6 +58,18 @@ def test_roofline_point_picks_the_binding_bound():
     assert bench.roofline_point(w5, 256, 3.4e8, hbm, fp32)["bound"] == "alu"           # fused: the sine
 
 
+def test_compact_summary_marks_target_points():
+    sweep = {"1": {"env_steps_per_sec": 1.0e9, "frac": 0.7, "meets_60pct": True, "target_point": True},
+             "4": {"env_steps_per_sec": 2.0e9, "frac": 0.3, "meets_60pct": False, "target_point": True},
+             "16": {"env_steps_per_sec": 3.0e9, "frac": 0.1, "meets_60pct": False, "target_point": False}}
+    out = bench.compact_summary({"w": {"k_sweep": sweep}}, "cfg2", {"1000": {"env_steps_per_sec": 2.5e11, "frac": 0.85, "meets_60pct": True, "target_point": True}})
+    assert out == ["w K1=1e+09/0.70* K4=2e+09/0.30! K16=3e+09/0.10", "cfg2 K1000=2.5e+11/0.85*"]
+    # every side pass names a workload of the table or one of the extra (non-task) ones, and the target table only names side passes
+    keys = {k for k, _, _ in bench.SIDE_PASSES}
+    assert all(w in inputs.WORKLOADS or w in bench.EXTRA_WORKLOADS for _, w, _ in bench.SIDE_PASSES)
+    assert set(bench.TARGET_POINTS) - {"cfg2"} <= keys
+
+
 def test_reference_arm_other_ranks_do_nothing():
     env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1"],

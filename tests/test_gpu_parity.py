@@ -418,3 +418,20 @@ def test_rollout_records_into_a_cuda_graph_captured_by_the_caller():
         for k in ("obs", "act", "rew", "done"):
             assert_same_bits(to_np(out[k]), ref[k], "graph replay %d %s" % (replay, k))
         assert_same_bits(to_np(sim.state()), orc.state, "state after replay")
+
+
+def test_calls_with_another_device_current_are_refused():
+    """A handle belongs to the device it was created on; with another device current every call that would touch
+    its buffers returns SIM_ESTATE and enqueues nothing (needs two GPUs; skipped on a single-GPU machine)."""
+    torch = torch_cuda()
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two CUDA devices")
+    sim = binding.Sim(oracle.CARTPOLE, 64, 4, 0, device="cuda:0")
+    L = binding.lib()
+    with torch.cuda.device(1):
+        assert L.sim_reset(sim.h) == binding.SIM_ESTATE
+        assert L.sim_rollout(sim.h, 4, 4, None, None, None, None, None) == binding.SIM_ESTATE
+        buf = torch.zeros(64 * 4, dtype=torch.float32, device="cuda:0")
+        assert L.sim_get_state(sim.h, buf.data_ptr()) == binding.SIM_ESTATE
+    with torch.cuda.device(0):
+        assert L.sim_reset(sim.h) == binding.SIM_OK
